@@ -1,0 +1,237 @@
+/*
+ * specscale.h - C ABI of the B200 (sm_100a) hot path of speculative expand-verify-select search:
+ *
+ *   ss_dedup_paths      computation deduplication of identical candidate paths
+ *   ss_tree_attention   attention of candidate paths over a paged bf16 KV pool described by a
+ *                       prefix / branch / leaf tree (decode: 1 query token per path; verification: a causal
+ *                       multi-token step per path)
+ *   ss_topk_prune       selection of the surviving candidates by score
+ *
+ * Conventions (all entry points)
+ *   - Unless a parameter says "host", every pointer is a DEVICE pointer owned by the caller.  The library
+ *     allocates no memory and keeps no state between calls; scratch comes from a caller-provided workspace
+ *     whose size is returned by a pure host query (no CUDA call inside the query).
+ *   - All work is enqueued on the caller's CUDA stream, passed as void* (a cudaStream_t; NULL = the legacy
+ *     default stream).  No entry point synchronises the host with the device, except
+ *     ss_last_device_status, which exists to do exactly that.
+ *   - Every function returns an int32_t status.  Argument errors are detected on the host before any launch.
+ *     Errors that only the device can see (an unsupported tree shape, a workspace that turns out too small
+ *     for the tree, a bounded wait that expired) are recorded in the first bytes of the workspace and read
+ *     back with ss_last_device_status; a call that recorded such an error leaves its outputs unspecified
+ *     but never reads or writes outside the buffers it was given (as far as the index arrays are valid;
+ *     SS_FLAG_VALIDATE makes the library check them too).
+ *   - No exceptions, no abort, no device printf.
+ */
+#ifndef SPECSCALE_H_
+#define SPECSCALE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- status codes ------------------------------------------------------------------------------------ */
+#define SS_OK 0
+#define SS_ERR_INVALID_ARG 1        /* null pointer, negative size, inconsistent scalar arguments            */
+#define SS_ERR_UNSUPPORTED 2        /* head_dim != 128, page_size != 16, Hq % Hkv != 0, Hq/Hkv > 128,
+                                       pool rows not contiguous, tree deeper than SS_MAX_DEPTH, a shared
+                                       (non-leaf) node whose length is not a multiple of the page size      */
+#define SS_ERR_WORKSPACE_TOO_SMALL 3
+#define SS_ERR_CUDA 4               /* a CUDA runtime / driver call failed (launch, tensor-map encode)       */
+#define SS_ERR_BAD_INPUT 5          /* SS_FLAG_VALIDATE found an out-of-range index in a descriptor array    */
+#define SS_ERR_TIMEOUT 6            /* a bounded device-side wait expired; the kernel drained and returned   */
+
+/* ---- flags --------------------------------------------------------------------------------------------- */
+#define SS_FLAG_VALIDATE 0x1u       /* check every index array on the device before it is used               */
+#define SS_FLAG_FORCE_GENERIC 0x2u  /* attention: run every path through the simple one-row-per-warp kernel
+                                       (no sharing, no tensor cores); a debugging aid and a second opinion  */
+#define SS_FLAG_NO_TCGEN05 0x4u     /* attention: keep the plan but run shared-node / verification tiles on
+                                       the simple kernel instead of the tcgen05 kernel                      */
+#define SS_FLAG_WEAK_HASH 0x8u      /* dedup: truncate the path hash to 8 bits so that collisions are common;
+                                       results must not change (tests the exact-comparison path)            */
+
+#define SS_MAX_DEPTH 16             /* maximum number of nodes on a root-to-leaf chain                       */
+
+const char* ss_status_string(int32_t status);   /* host; static string, never NULL */
+
+/* Reads the status word that the last call using this workspace recorded on the device.  Copies 4 bytes
+ * device->host on `stream` and waits for that stream.  *out_status (host) receives SS_OK or an SS_ERR_*.
+ * Returns SS_OK if the read itself worked. */
+int32_t ss_last_device_status(const void* workspace, void* stream, int32_t* out_status);
+
+/* =========================================================================================================
+ * ss_dedup_paths - computation deduplication.
+ *
+ * Paper: Section "Computation Deduplication" - candidates "with identical input sequences" share one
+ * forward pass; the number of logical candidates a sequence stands for is its "potential" size, and
+ * sampled continuations are grouped by equality with one child per group whose potential is the group's
+ * cardinality (worked example: three equal samples and one different -> potentials 3 and 1).
+ *
+ * Two logical paths i, j are duplicates iff ctx_key[i] == ctx_key[j] and their token-id sequences are equal
+ * (same length, same ids).  Hashing is internal: collisions never change a result (equal-hash candidates are
+ * compared token by token).
+ *
+ *   tok_ids        int32 [tok_offsets[n_paths]]   token ids, CSR by path
+ *   tok_offsets    int64 [n_paths+1]              ascending, tok_offsets[0] may be any value >= 0
+ *   ctx_key        int64 [n_paths] or NULL        opaque context that must also match (parent node, mode...)
+ *   slot_in        int32 [n_paths] or NULL        KV slot (e.g. leaf node id) of each logical path
+ *   n_paths        host, >= 0 (0: only *num_unique_out = 0 is written)
+ *   flags          0 or SS_FLAG_WEAK_HASH
+ *   canon_out          int32 [n_paths]   smallest index whose (ctx_key, sequence) equals path i's
+ *   path_to_unique_out int32 [n_paths]   rank of canon_out[i] among the unique paths (ascending index order)
+ *   unique_paths_out   int32 [n_paths]   first U entries valid: the unique paths, ascending
+ *   multiplicity_out   int32 [n_paths]   first U entries valid: group sizes (the "potential" sizes)
+ *   slot_out           int32 [n_paths] or NULL (must be NULL iff slot_in is NULL): slot_in[canon_out[i]]
+ *   num_unique_out     int32 [1]         U
+ *   workspace      >= ss_dedup_workspace_bytes(n_paths) bytes, 256-byte aligned
+ *
+ * Outputs are unique (no ordering freedom) and bit-exact with the plain std::map definition.
+ * Errors: SS_ERR_INVALID_ARG, SS_ERR_WORKSPACE_TOO_SMALL, SS_ERR_CUDA.
+ * ======================================================================================================= */
+int32_t ss_dedup_workspace_bytes(int32_t n_paths, size_t* out_bytes /* host */);
+int32_t ss_dedup_paths(const int32_t* tok_ids, const int64_t* tok_offsets, const int64_t* ctx_key,
+                       const int32_t* slot_in, int32_t n_paths, uint32_t flags, int32_t* canon_out,
+                       int32_t* path_to_unique_out, int32_t* unique_paths_out, int32_t* multiplicity_out,
+                       int32_t* slot_out, int32_t* num_unique_out, void* workspace, size_t workspace_bytes,
+                       void* stream);
+
+/* =========================================================================================================
+ * ss_tree_attention - attention over a tree of candidate paths that share KV prefixes.
+ *
+ * Paper: the serving substrate of Section "Experimental Setup" (paged attention, prefix KV caching and
+ * sharing, fused attention kernels), used for the decode phase of expansion (Section "LLM Inference and
+ * Serving") and for verification, which "is a prefill-only workload" over short steps (Section "Lazy
+ * Verification").  The paper prints no formula; the operation is standard softmax attention:
+ *
+ *   for path p with KV sequence = concatenation of its nodes root -> leaf (length L), step length T:
+ *     query token t (0 <= t < T), q head h, kv head g = h / (Hq/Hkv):
+ *       s_j = sm_scale * <q[t,h,:], K[j,g,:]>            for keys j <= L - T + t  (bottom-right causal)
+ *       out[t,h,:] = sum_j softmax(s)_j V[j,g,:]         lse[t,h] = ln sum_j exp(s_j)   (natural log)
+ *     no visible key  =>  out = 0, lse = -inf.
+ *
+ * The step's own keys/values are expected to be in the pool already (they are the last T tokens of the
+ * path's leaf node; appending them is outside this call).  Positional encoding is outside this call.
+ *
+ * Tree: nodes are numbered parents-before-children; node n holds node_kv_len[n] tokens in the pages
+ * node_pages[node_page_offsets[n] .. node_page_offsets[n+1]) (16 tokens each; only the last page may be
+ * partly filled; slots past the length are never read into a result).  A node that lies on the chain of
+ * several paths is read once for all of them.  Paths are the UNIQUE paths (after ss_dedup_paths) in tree
+ * order: the paths below any node are contiguous.  Every node with more than one path below it must hold a
+ * multiple of 16 tokens.
+ *
+ * KV pool: bf16.  Element (page, kv head, token-in-page, dim) of K is
+ *   k_pool[page*kv_page_stride + head*kv_head_stride + token*kv_token_stride + dim]   (strides in elements)
+ * and likewise for v_pool.  Supported: kv_token_stride == head_dim (each (page, head) block is 16 contiguous
+ * rows of 256 bytes), kv_page_stride and kv_head_stride multiples of 128 elements, k_pool and v_pool 256-byte
+ * aligned.  The recommended pool is one allocation laid out [page][K|V][kv head][16][128].
+ *
+ * q   bf16 [total_q][Hq][128], rows of path p are q_offsets[p] .. q_offsets[p+1]-1, 16-byte aligned
+ * out bf16 [total_q][Hq][128]   (fp32 accumulation, rounded to nearest even), 16-byte aligned
+ * lse fp32 [total_q][Hq]        or NULL
+ *
+ * Accuracy contract (inputs ~N(0,1) in bf16): |out - exact| <= 2e-2 max, 2e-3 mean; |lse - exact| <= 1e-3.
+ *
+ * Errors (host): SS_ERR_INVALID_ARG, SS_ERR_UNSUPPORTED, SS_ERR_WORKSPACE_TOO_SMALL, SS_ERR_CUDA.
+ * Errors (device, via ss_last_device_status): SS_ERR_UNSUPPORTED (depth, node length), SS_ERR_BAD_INPUT
+ * (with SS_FLAG_VALIDATE), SS_ERR_WORKSPACE_TOO_SMALL (hints below were too low), SS_ERR_TIMEOUT.
+ * ======================================================================================================= */
+typedef struct ss_attn_desc {
+  uint32_t struct_size;              /* = sizeof(ss_attn_desc_t) */
+  uint32_t flags;                    /* SS_FLAG_* */
+  int32_t num_q_heads, num_kv_heads; /* Hq % Hkv == 0 */
+  int32_t head_dim, page_size;       /* 128, 16 */
+  float sm_scale;                    /* 0 => 1/sqrt(head_dim) */
+  int32_t reserved0;
+  const void* k_pool;                /* bf16 */
+  const void* v_pool;                /* bf16 */
+  int64_t num_pages;                 /* pages addressable through k_pool / v_pool */
+  int64_t kv_page_stride, kv_head_stride, kv_token_stride; /* elements */
+  /* ---- tree ---- */
+  int32_t num_nodes;
+  int32_t reserved1;
+  const int32_t* node_parent;        /* [num_nodes]  -1 for a root */
+  const int32_t* node_kv_len;        /* [num_nodes]  >= 0 */
+  const int64_t* node_page_offsets;  /* [num_nodes+1] */
+  const int32_t* node_pages;         /* [total_node_pages] physical page ids */
+  int64_t total_node_pages;          /* host copy of node_page_offsets[num_nodes] (an upper bound is fine) */
+  /* ---- paths ---- */
+  int32_t num_paths;                 /* capacity of the per-path arrays */
+  int32_t reserved2;
+  const int32_t* num_paths_dev;      /* NULL, or a device scalar <= num_paths holding the live path count
+                                        (e.g. num_unique_out of ss_dedup_paths): no host sync needed between
+                                        the two calls */
+  const int32_t* path_leaf_node;     /* [num_paths] */
+  const int32_t* path_q_len;         /* [num_paths] T >= 1 */
+  const int64_t* q_offsets;          /* [num_paths+1] */
+  int64_t total_q;                   /* host upper bound of q_offsets[live paths] */
+  /* ---- sizing hints (host scalars; 0 = use the safe default; tight values shrink the workspace) ---- */
+  int32_t max_depth;                 /* nodes on the longest chain; default SS_MAX_DEPTH */
+  int32_t max_decode_paths;          /* paths with T == 1; default num_paths */
+  /* ---- data ---- */
+  const void* q;
+  void* out;
+  float* lse;
+} ss_attn_desc_t;
+
+int32_t ss_tree_attention_workspace_bytes(const ss_attn_desc_t* desc /* host */, size_t* out_bytes /* host */);
+int32_t ss_tree_attention(const ss_attn_desc_t* desc /* host */, void* workspace, size_t workspace_bytes,
+                          void* stream);
+
+/* =========================================================================================================
+ * ss_topk_prune - keep the k best-scored candidates of every problem.
+ *
+ * Paper: Section "Early Pruning of Search Tree" - a candidate whose score ranks below the top-k cannot be
+ * part of the final top-k and is pruned; Section "Test-Time Scaling" - top-k = N / M (beam size / width).
+ * Ordering: score descending, ties to the lower index (the paper cannot distinguish equal scores); -0.0 equals
+ * +0.0; NaN ranks below every number.  The result is unique.
+ *
+ *   scores        fp32 [n_total]
+ *   seg_offsets   int32 [n_segments+1]  ascending; segment s = candidates seg_offsets[s] .. seg_offsets[s+1]-1
+ *   n_segments    host >= 0;  n_total host >= seg_offsets[n_segments];  k host >= 1
+ *   survivors_out int32 [n_segments][k]  global candidate indices, best first, -1 padded when a segment has
+ *                 fewer than k candidates
+ *   keep_out      uint8 [n_total]        1 iff the candidate survives (entries outside every segment: 0)
+ *   workspace     >= ss_topk_workspace_bytes(n_total) bytes, 256-byte aligned
+ * Errors: SS_ERR_INVALID_ARG, SS_ERR_WORKSPACE_TOO_SMALL, SS_ERR_CUDA.
+ * ======================================================================================================= */
+int32_t ss_topk_workspace_bytes(int32_t n_total, size_t* out_bytes /* host */);
+int32_t ss_topk_prune(const float* scores, const int32_t* seg_offsets, int32_t n_segments, int32_t n_total,
+                      int32_t k, int32_t* survivors_out, uint8_t* keep_out, void* workspace,
+                      size_t workspace_bytes, void* stream);
+
+/* =========================================================================================================
+ * Diagnostics
+ * ======================================================================================================= */
+/* Number of kernels this library has launched in this process since it was loaded (host counter). */
+int64_t ss_launch_count(void);
+
+/* Per-phase timing of ss_tree_attention with CUDA events (diagnostics; no paper counterpart).
+ * While enabled, every ss_tree_attention call records events on its stream around each phase
+ * (SS_PHASE_*); the events come from a fixed pool created on first use (calls beyond the pool are not timed).
+ * ss_profile_read waits for the recorded events, adds up the milliseconds and the number of timed calls per
+ * phase into the host arrays (each SS_NUM_PHASES long; either may be NULL) and clears the record.
+ * Not thread-safe; meant for a benchmark harness. */
+#define SS_PHASE_PLAN 0
+#define SS_PHASE_TILES 1      /* tcgen05 tile items: shared-node (stacked decode rows) and verification tiles */
+#define SS_PHASE_LEAVES 2     /* bandwidth-bound decode-leaf items */
+#define SS_PHASE_GENERIC 3
+#define SS_PHASE_MERGE 4
+#define SS_NUM_PHASES 5
+int32_t ss_profile_enable(int32_t on);
+int32_t ss_profile_read(float* phase_ms /* host */, int64_t* phase_calls /* host */);
+
+/* One 128 x N x K bf16 tile product on the tcgen05 tensor cores, C[128][N] (fp32, row-major) = A[128][K] *
+ * op(B), with the same shared-memory descriptors and TMEM read-out as the attention kernel.
+ *   b_is_mn_major == 0: B is [N][K] row-major (the K-operand form, like keys);  C = A * B^T
+ *   b_is_mn_major == 1: B is [K][N] row-major (the value form);                 C = A * B
+ * N in {64, 128}, K a multiple of 64 and <= 256.  No paper counterpart: a self-test of the tensor-core
+ * plumbing.  status_out: device int32[1], receives SS_OK or SS_ERR_TIMEOUT. */
+int32_t ss_debug_umma_tile(const void* a_bf16, const void* b_bf16, float* c, int32_t n, int32_t k,
+                           int32_t b_is_mn_major, int32_t* status_out, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPECSCALE_H_ */

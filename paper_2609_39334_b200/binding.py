@@ -1,0 +1,230 @@
+"""Thin ctypes binding of libspecscale.so - argument marshalling only.
+
+The functions carry the names of the C ABI (include/specscale.h).  Tensors are torch tensors that already live on
+the GPU; torch provides device memory and streams and nothing else.  There is no CPU fallback: if the CUDA
+library is missing, loading fails with an error.
+"""
+from __future__ import annotations
+
+import ctypes
+import math
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libspecscale.so")
+
+SS_OK = 0
+SS_ERR_INVALID_ARG = 1
+SS_ERR_UNSUPPORTED = 2
+SS_ERR_WORKSPACE_TOO_SMALL = 3
+SS_ERR_CUDA = 4
+SS_ERR_BAD_INPUT = 5
+SS_ERR_TIMEOUT = 6
+SS_FLAG_VALIDATE = 0x1
+SS_FLAG_FORCE_GENERIC = 0x2
+SS_FLAG_NO_TCGEN05 = 0x4
+SS_FLAG_WEAK_HASH = 0x8
+SS_MAX_DEPTH = 16
+
+EXPORTS = [
+    "ss_status_string", "ss_last_device_status", "ss_dedup_workspace_bytes", "ss_dedup_paths",
+    "ss_tree_attention_workspace_bytes", "ss_tree_attention", "ss_topk_workspace_bytes", "ss_topk_prune",
+    "ss_launch_count", "ss_debug_umma_tile", "ss_profile_enable", "ss_profile_read",
+]
+PHASES = ["plan", "tiles", "leaves", "generic", "merge"]
+
+
+class SpecScaleError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+class ss_attn_desc_t(ctypes.Structure):
+    _fields_ = [
+        ("struct_size", ctypes.c_uint32), ("flags", ctypes.c_uint32),
+        ("num_q_heads", ctypes.c_int32), ("num_kv_heads", ctypes.c_int32),
+        ("head_dim", ctypes.c_int32), ("page_size", ctypes.c_int32),
+        ("sm_scale", ctypes.c_float), ("reserved0", ctypes.c_int32),
+        ("k_pool", ctypes.c_void_p), ("v_pool", ctypes.c_void_p),
+        ("num_pages", ctypes.c_int64),
+        ("kv_page_stride", ctypes.c_int64), ("kv_head_stride", ctypes.c_int64), ("kv_token_stride", ctypes.c_int64),
+        ("num_nodes", ctypes.c_int32), ("reserved1", ctypes.c_int32),
+        ("node_parent", ctypes.c_void_p), ("node_kv_len", ctypes.c_void_p),
+        ("node_page_offsets", ctypes.c_void_p), ("node_pages", ctypes.c_void_p),
+        ("total_node_pages", ctypes.c_int64),
+        ("num_paths", ctypes.c_int32), ("reserved2", ctypes.c_int32),
+        ("num_paths_dev", ctypes.c_void_p), ("path_leaf_node", ctypes.c_void_p), ("path_q_len", ctypes.c_void_p),
+        ("q_offsets", ctypes.c_void_p), ("total_q", ctypes.c_int64),
+        ("max_depth", ctypes.c_int32), ("max_decode_paths", ctypes.c_int32),
+        ("q", ctypes.c_void_p), ("out", ctypes.c_void_p), ("lse", ctypes.c_void_p),
+    ]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads the CUDA library; raises if it has not been built (there is no other implementation)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2609_39334_b200.build`; "
+                               "there is no CPU fallback")
+        L = ctypes.CDLL(LIB_PATH)
+        L.ss_status_string.restype = ctypes.c_char_p
+        L.ss_status_string.argtypes = [ctypes.c_int32]
+        L.ss_launch_count.restype = ctypes.c_int64
+        for name in EXPORTS:
+            if name not in ("ss_status_string", "ss_launch_count"):
+                getattr(L, name).restype = ctypes.c_int32
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().ss_status_string(int(status)).decode()
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    if t is None:
+        return ctypes.c_void_p(0)
+    assert t.is_cuda and t.is_contiguous(), "device-resident contiguous tensors only"
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream))
+
+
+def _check(rc: int, where: str):
+    if rc != SS_OK:
+        raise SpecScaleError(rc, where)
+
+
+def alloc_workspace(nbytes: int, device) -> torch.Tensor:
+    """Device scratch for one call (256-byte aligned: torch's allocator aligns to 512)."""
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+def ss_launch_count() -> int:
+    return int(lib().ss_launch_count())
+
+
+def ss_last_device_status(workspace: torch.Tensor, stream=None) -> int:
+    out = ctypes.c_int32(-1)
+    _check(lib().ss_last_device_status(_ptr(workspace), _stream(stream), ctypes.byref(out)), "ss_last_device_status")
+    return int(out.value)
+
+
+# ---------------------------------------------------------------------------------------------------------
+def ss_dedup_workspace_bytes(n_paths: int) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().ss_dedup_workspace_bytes(ctypes.c_int32(n_paths), ctypes.byref(out)), "ss_dedup_workspace_bytes")
+    return int(out.value)
+
+
+def ss_dedup_paths(tok_ids, tok_offsets, ctx_key, slot_in, n_paths, flags, canon_out, path_to_unique_out,
+                   unique_paths_out, multiplicity_out, slot_out, num_unique_out, workspace, stream=None,
+                   check=True) -> int:
+    rc = lib().ss_dedup_paths(_ptr(tok_ids), _ptr(tok_offsets), _ptr(ctx_key), _ptr(slot_in), ctypes.c_int32(n_paths),
+                              ctypes.c_uint32(flags), _ptr(canon_out), _ptr(path_to_unique_out),
+                              _ptr(unique_paths_out), _ptr(multiplicity_out), _ptr(slot_out), _ptr(num_unique_out),
+                              _ptr(workspace), ctypes.c_size_t(workspace.numel() if workspace is not None else 0),
+                              _stream(stream))
+    if check:
+        _check(rc, "ss_dedup_paths")
+    return rc
+
+
+# ---------------------------------------------------------------------------------------------------------
+def make_attn_desc(*, num_q_heads, num_kv_heads, kv_pool=None, k_pool=None, v_pool=None, num_pages=None,
+                   kv_page_stride=None, kv_head_stride=None, kv_token_stride=None, node_parent, node_kv_len,
+                   node_page_offsets, node_pages, total_node_pages, path_leaf_node, path_q_len, q_offsets, total_q,
+                   q, out, lse=None, num_paths=None, num_paths_dev=None, sm_scale=0.0, flags=0, max_depth=0,
+                   max_decode_paths=0, head_dim=128, page_size=16) -> ss_attn_desc_t:
+    """Fills the descriptor.  `kv_pool` is the recommended single allocation [page][2][Hkv][16][128]; otherwise
+    give k_pool / v_pool tensors and the element strides."""
+    d = ss_attn_desc_t()
+    d.struct_size = ctypes.sizeof(ss_attn_desc_t)
+    d.flags = flags
+    d.num_q_heads, d.num_kv_heads, d.head_dim, d.page_size = num_q_heads, num_kv_heads, head_dim, page_size
+    d.sm_scale = float(sm_scale)
+    if kv_pool is not None:
+        assert kv_pool.dim() == 5 and kv_pool.is_contiguous() and kv_pool.dtype == torch.bfloat16
+        blk = num_kv_heads * page_size * head_dim
+        d.k_pool = kv_pool.data_ptr()
+        d.v_pool = kv_pool.data_ptr() + blk * 2
+        d.num_pages = kv_pool.shape[0]
+        d.kv_page_stride, d.kv_head_stride, d.kv_token_stride = 2 * blk, page_size * head_dim, head_dim
+    else:
+        d.k_pool, d.v_pool = k_pool.data_ptr(), v_pool.data_ptr()
+        d.num_pages = num_pages
+        d.kv_page_stride, d.kv_head_stride, d.kv_token_stride = kv_page_stride, kv_head_stride, kv_token_stride
+    d.num_nodes = int(node_parent.shape[0])
+    d.node_parent, d.node_kv_len = node_parent.data_ptr(), node_kv_len.data_ptr()
+    d.node_page_offsets, d.node_pages = node_page_offsets.data_ptr(), node_pages.data_ptr()
+    d.total_node_pages = int(total_node_pages)
+    d.num_paths = int(path_leaf_node.shape[0]) if num_paths is None else int(num_paths)
+    d.num_paths_dev = num_paths_dev.data_ptr() if num_paths_dev is not None else None
+    d.path_leaf_node, d.path_q_len, d.q_offsets = path_leaf_node.data_ptr(), path_q_len.data_ptr(), q_offsets.data_ptr()
+    d.total_q = int(total_q)
+    d.max_depth, d.max_decode_paths = int(max_depth), int(max_decode_paths)
+    d.q = q.data_ptr() if q is not None else None
+    d.out = out.data_ptr() if out is not None else None
+    d.lse = lse.data_ptr() if lse is not None else None
+    return d
+
+
+def ss_tree_attention_workspace_bytes(desc: ss_attn_desc_t) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().ss_tree_attention_workspace_bytes(ctypes.byref(desc), ctypes.byref(out)),
+           "ss_tree_attention_workspace_bytes")
+    return int(out.value)
+
+
+def ss_tree_attention(desc: ss_attn_desc_t, workspace: torch.Tensor, stream=None, check=True) -> int:
+    rc = lib().ss_tree_attention(ctypes.byref(desc), _ptr(workspace), ctypes.c_size_t(workspace.numel()),
+                                 _stream(stream))
+    if check:
+        _check(rc, "ss_tree_attention")
+    return rc
+
+
+# ---------------------------------------------------------------------------------------------------------
+def ss_topk_workspace_bytes(n_total: int) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().ss_topk_workspace_bytes(ctypes.c_int32(n_total), ctypes.byref(out)), "ss_topk_workspace_bytes")
+    return int(out.value)
+
+
+def ss_topk_prune(scores, seg_offsets, n_segments, n_total, k, survivors_out, keep_out, workspace, stream=None,
+                  check=True) -> int:
+    rc = lib().ss_topk_prune(_ptr(scores), _ptr(seg_offsets), ctypes.c_int32(n_segments), ctypes.c_int32(n_total),
+                             ctypes.c_int32(k), _ptr(survivors_out), _ptr(keep_out), _ptr(workspace),
+                             ctypes.c_size_t(workspace.numel() if workspace is not None else 0), _stream(stream))
+    if check:
+        _check(rc, "ss_topk_prune")
+    return rc
+
+
+def ss_debug_umma_tile(a, b, c, n, k, b_is_mn_major, status_out, stream=None) -> int:
+    return lib().ss_debug_umma_tile(_ptr(a), _ptr(b), _ptr(c), ctypes.c_int32(n), ctypes.c_int32(k),
+                                    ctypes.c_int32(b_is_mn_major), _ptr(status_out), _stream(stream))
+
+
+def ss_profile_enable(on: bool) -> None:
+    _check(lib().ss_profile_enable(ctypes.c_int32(1 if on else 0)), "ss_profile_enable")
+
+
+def ss_profile_read():
+    """-> ({phase: total ms}, {phase: timed calls}) since the last read."""
+    ms = (ctypes.c_float * len(PHASES))()
+    calls = (ctypes.c_int64 * len(PHASES))()
+    _check(lib().ss_profile_read(ms, calls), "ss_profile_read")
+    return {p: float(ms[i]) for i, p in enumerate(PHASES)}, {p: int(calls[i]) for i, p in enumerate(PHASES)}

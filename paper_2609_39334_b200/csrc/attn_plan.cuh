@@ -1,0 +1,105 @@
+// Plan structures of ss_tree_attention: how the tree of candidate paths is cut into kernel work items.
+//
+// Path classes
+//   DECODE   T == 1.  Level-split: every node on the chain that is shared (or is not this path's private
+//            leaf) is processed once for ALL decode tokens below it by stacked "tile items" (tensor cores),
+//            the path's private leaf by "leaf items" (bandwidth-bound kernel); the per-level partial results
+//            are combined by the log-sum-exp merge.
+//   CHAIN    T > 1 (a verification step).  A tile of up to 128 stacked rows (tokens x GQA group) of ONE path
+//            walks the path's whole KV chain root -> leaf in one pass (causal tail inside the leaf) and writes
+//            the final result: no partials.  Shared prefixes are re-used through L2.
+//   GENERIC  anything the fast kernels do not take (an inner chain node that is not a whole number of pages,
+//            a GQA group > 16 for decode, or SS_FLAG_FORCE_GENERIC): one warp per (query token, head).
+#pragma once
+#include "common.cuh"
+
+namespace ss {
+namespace attn {
+
+constexpr int kHeadDim = 128;
+constexpr int kPage = 16;
+constexpr int kTileRows = 128;          // stacked rows of one tile item
+constexpr int kKvTile = 64;             // keys per tensor-core step
+constexpr int kLeafChunk = 256;         // keys per leaf item (decode)
+constexpr int kMaxRootSplits = 8;       // KV splits of a root node when there are few tiles
+constexpr int kMinSplitLen = 512;       // a split is at least this many keys
+
+enum PathClass : int32_t { kClassDecode = 0, kClassChain = 1, kClassGeneric = 2 };
+enum ItemKind : int32_t { kItemStacked = 0, kItemChain = 1 };
+
+// One tile of stacked query rows against a KV source.  32 bytes.
+struct TileItem {
+  int32_t node;       // stacked: the shared node; chain: the path's leaf node
+  int32_t tok0;       // stacked: index into dec_tok[]; chain: first query row (global token index)
+  int32_t n_tok;      // tokens in the tile (rows = n_tok * G)
+  int32_t kind_g;     // kind << 16 | kv head
+  int32_t kv_begin;   // token range [kv_begin, kv_end) of the source's virtual key sequence
+  int32_t kv_end;
+  int32_t limit0;     // keys visible to the tile's first token; token i sees limit0 + i * (kind == chain)
+  int32_t slot_off;   // stacked: partial slot relative to the token's slot base; chain: -1 (final output)
+};
+
+// One chunk of a decode path's private leaf.  32 bytes.
+struct LeafItem {
+  int32_t q_row;      // global query token index
+  int32_t node;       // leaf node
+  int32_t g;          // kv head
+  int32_t kv_begin;   // token range inside the leaf
+  int32_t kv_end;
+  int32_t slot;       // absolute partial slot
+  int32_t pad0, pad1;
+};
+
+struct PlanHeader {       // first bytes of the workspace; status MUST be the first word
+  int32_t status;
+  int32_t live_paths;
+  int32_t n_dec;          // decode tokens
+  int32_t n_tile_items;
+  int32_t n_leaf_items;
+  int32_t n_slots;
+  int32_t n_generic_rows; // > 0 if any path is GENERIC
+  int32_t tile_counter;   // work-stealing counters (reset by the planner)
+  int32_t leaf_counter;
+  int32_t pad[7];
+};
+
+struct Caps {             // host-computed capacities of the plan arrays
+  int32_t dec, tile_items, leaf_items;
+  int64_t slots;
+};
+
+// Everything a kernel needs, passed by value.
+struct Params {
+  int32_t Hq, Hkv, G, tok_per_tile;
+  float scale, scale_log2;
+  uint32_t flags;
+  const __nv_bfloat16 *k_pool, *v_pool;
+  int64_t num_pages, page_stride, head_stride, token_stride;
+  int32_t num_nodes;
+  const int32_t *node_parent, *node_kv_len;
+  const int64_t* node_page_offsets;
+  const int32_t* node_pages;
+  int64_t total_node_pages;
+  int32_t num_paths;
+  const int32_t *num_paths_dev, *path_leaf_node, *path_q_len;
+  const int64_t* q_offsets;
+  int64_t total_q;
+  const __nv_bfloat16* q;
+  __nv_bfloat16* out;
+  float* lse;
+  int32_t target_tiles;      // the planner splits root nodes until about this many tile items exist
+  Caps caps;
+  // ---- workspace regions ----
+  PlanHeader* hdr;
+  int32_t *node_start, *node_depth, *node_first, *node_last, *node_npaths, *node_ndec, *node_own_slots,
+      *node_level_off, *node_item_base, *node_splits, *node_split_len;
+  int32_t *path_class, *path_kv_len, *path_dec_rank, *path_scan;
+  int32_t *dec_tok, *dec_slot_base;
+  TileItem* tile_items;
+  LeafItem* leaf_items;
+  float* part_o;             // [slots][Hq][128]
+  float* part_lse;           // [slots][Hq]
+};
+
+}  // namespace attn
+}  // namespace ss

@@ -1,0 +1,324 @@
+// ss_dedup_paths: computation deduplication of candidate paths (paper, Section "Computation Deduplication").
+//
+// Pipeline (all on the caller's stream, no host synchronisation):
+//   1. hash      one warp per path: 64-bit hash of (ctx_key, length, token ids); lanes stride over the tokens,
+//                each token is mixed with its position, lane sums are combined with shuffles
+//   2. sort      LSD radix sort (8-bit digits, 4 passes) of (top 32 hash bits, path index); stable, so equal
+//                keys stay in ascending index order
+//   3. match     one warp per sorted position: binary-search the start of its equal-key run, then look for the
+//                first earlier run member whose full 64-bit hash, ctx_key, length AND token ids are equal
+//                (token ids compared cooperatively by the warp) -> canon
+//   4. compact   exclusive scan of (canon[i] == i) in index order -> ranks; unique list, multiplicities
+//                (integer atomics: order-independent), path_to_unique, slot remap
+// Hash collisions only cost time: equality is always decided on the token ids themselves.
+#include "common.cuh"
+
+namespace ss {
+namespace dedup {
+
+constexpr int kSortThreads = 256;
+constexpr int kSortItems = 8;                       // rounds per tile
+constexpr int kSortTile = kSortThreads * kSortItems;
+constexpr int kWarpsPerSortBlock = kSortThreads / 32;
+
+__device__ __forceinline__ uint64_t mix64(uint64_t x) {   // splitmix64 finaliser
+  x ^= x >> 30; x *= 0xbf58476d1ce4e5b9ull;
+  x ^= x >> 27; x *= 0x94d049bb133111ebull;
+  x ^= x >> 31;
+  return x;
+}
+
+__global__ void hash_kernel(const int32_t* __restrict__ tok_ids, const int64_t* __restrict__ tok_offsets,
+                            const int64_t* __restrict__ ctx_key, int n, uint32_t weak, uint64_t* __restrict__ hash64,
+                            uint32_t* __restrict__ keys, uint32_t* __restrict__ idx) {
+  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (warp >= n) return;
+  const int64_t lo = tok_offsets[warp], hi = tok_offsets[warp + 1];
+  uint64_t acc = 0;
+  for (int64_t j = lo + lane; j < hi; j += 32) {
+    const uint64_t t = static_cast<uint32_t>(tok_ids[j]);
+    acc += mix64(t * 0x9e3779b97f4a7c15ull + static_cast<uint64_t>(j - lo + 1) * 0xd1b54a32d192ed03ull);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  if (lane == 0) {
+    uint64_t h = mix64(acc ^ mix64(static_cast<uint64_t>(hi - lo) + 0x632be59bd9b4e019ull));
+    if (ctx_key) h = mix64(h ^ mix64(static_cast<uint64_t>(ctx_key[warp]) + 0x2545f4914f6cdd1dull));
+    if (weak) h &= 0xffull;                     // SS_FLAG_WEAK_HASH: force collisions
+    hash64[warp] = h;
+    keys[warp] = weak ? static_cast<uint32_t>(h) : static_cast<uint32_t>(h >> 32);
+    idx[warp] = warp;
+  }
+}
+
+// ---- radix sort pass -------------------------------------------------------------------------------------
+__global__ void rs_hist(const uint32_t* __restrict__ keys, int n, int shift, int num_tiles, uint32_t* __restrict__ hist) {
+  __shared__ uint32_t cnt[256];
+  cnt[threadIdx.x] = 0;
+  __syncthreads();
+  const int base = blockIdx.x * kSortTile;
+  for (int r = 0; r < kSortItems; ++r) {
+    const int i = base + r * kSortThreads + threadIdx.x;
+    if (i < n) atomicAdd(&cnt[(keys[i] >> shift) & 255u], 1u);
+  }
+  __syncthreads();
+  hist[threadIdx.x * num_tiles + blockIdx.x] = cnt[threadIdx.x];
+}
+
+// In-place exclusive sum scan of `count` uint32 by one block (looping with a carry).
+__global__ void scan_u32_single_block(uint32_t* __restrict__ data, int count) {
+  __shared__ uint32_t warp_tot[32];
+  __shared__ uint32_t carry_s;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  if (threadIdx.x == 0) carry_s = 0;
+  __syncthreads();
+  for (int base = 0; base < count; base += blockDim.x) {
+    const int i = base + threadIdx.x;
+    const uint32_t v = i < count ? data[i] : 0u;
+    uint32_t x = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t y = __shfl_up_sync(0xffffffffu, x, o);
+      if (lane >= o) x += y;
+    }
+    if (lane == 31) warp_tot[warp] = x;
+    __syncthreads();
+    if (warp == 0) {
+      uint32_t t = lane < nw ? warp_tot[lane] : 0u;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t y = __shfl_up_sync(0xffffffffu, t, o);
+        if (lane >= o) t += y;
+      }
+      warp_tot[lane] = t;                         // inclusive totals of warps
+    }
+    __syncthreads();
+    const uint32_t carry = carry_s;
+    const uint32_t before = carry + (warp ? warp_tot[warp - 1] : 0u) + x - v;
+    if (i < count) data[i] = before;
+    __syncthreads();
+    if (threadIdx.x == blockDim.x - 1) carry_s = before + v;
+    __syncthreads();
+  }
+}
+
+__global__ void rs_scatter(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict__ idx_in,
+                           uint32_t* __restrict__ keys_out, uint32_t* __restrict__ idx_out, int n, int shift,
+                           int num_tiles, const uint32_t* __restrict__ hist) {
+  __shared__ uint32_t base[256];
+  __shared__ uint32_t wc[kWarpsPerSortBlock][256];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  base[threadIdx.x] = hist[threadIdx.x * num_tiles + blockIdx.x];
+#pragma unroll
+  for (int w = 0; w < kWarpsPerSortBlock; ++w) wc[w][threadIdx.x] = 0;
+  __syncthreads();
+  const int tile_base = blockIdx.x * kSortTile;
+  for (int r = 0; r < kSortItems; ++r) {
+    const int i = tile_base + r * kSortThreads + threadIdx.x;
+    const bool valid = i < n;
+    uint32_t key = 0, id = 0;
+    if (valid) { key = keys_in[i]; id = idx_in[i]; }
+    const uint32_t digit = valid ? ((key >> shift) & 255u) : 256u;
+    const uint32_t peers = __match_any_sync(0xffffffffu, digit);
+    const uint32_t rank = __popc(peers & ((1u << lane) - 1u));
+    if (valid && rank == 0) wc[warp][digit] = __popc(peers);
+    __syncthreads();
+    if (valid) {
+      uint32_t off = base[digit] + rank;
+      for (int w = 0; w < warp; ++w) off += wc[w][digit];
+      keys_out[off] = key;
+      idx_out[off] = id;
+    }
+    __syncthreads();
+    {
+      uint32_t tot = 0;
+#pragma unroll
+      for (int w = 0; w < kWarpsPerSortBlock; ++w) { tot += wc[w][threadIdx.x]; wc[w][threadIdx.x] = 0; }
+      base[threadIdx.x] += tot;
+    }
+    __syncthreads();
+  }
+}
+
+// ---- exact matching inside equal-key runs ---------------------------------------------------------------
+__global__ void match_kernel(const uint32_t* __restrict__ keys, const uint32_t* __restrict__ idx, int n,
+                             const uint64_t* __restrict__ hash64, const int32_t* __restrict__ tok_ids,
+                             const int64_t* __restrict__ tok_offsets, const int64_t* __restrict__ ctx_key,
+                             int32_t* __restrict__ canon_out) {
+  const int s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (s >= n) return;
+  const uint32_t key = keys[s];
+  const int i = static_cast<int>(idx[s]);
+  // start of the run of equal keys (lower bound)
+  int lo = 0, hi = s;
+  while (lo < hi) {
+    const int mid = (lo + hi) >> 1;
+    if (keys[mid] < key) lo = mid + 1; else hi = mid;
+  }
+  const uint64_t hi_ = hash64[i];
+  const int64_t a0 = tok_offsets[i], alen = tok_offsets[i + 1] - a0;
+  const int64_t actx = ctx_key ? ctx_key[i] : 0;
+  int canon = i;
+  for (int b = lo; b < s && canon == i; b += 32) {
+    const int t = b + lane;
+    bool cand = false;
+    int j = 0;
+    if (t < s) {
+      j = static_cast<int>(idx[t]);
+      cand = hash64[j] == hi_ && (tok_offsets[j + 1] - tok_offsets[j]) == alen && (ctx_key ? ctx_key[j] : 0) == actx;
+    }
+    uint32_t m = __ballot_sync(0xffffffffu, cand);
+    while (m) {
+      const int src = __ffs(m) - 1;
+      m &= m - 1;
+      const int jj = __shfl_sync(0xffffffffu, j, src);
+      const int64_t b0 = tok_offsets[jj];
+      bool same = true;
+      for (int64_t p = 0; p < alen && same; p += 32) {
+        const int64_t q = p + lane;
+        const bool eq = q < alen ? (tok_ids[a0 + q] == tok_ids[b0 + q]) : true;
+        same = __all_sync(0xffffffffu, eq);
+      }
+      if (same) { canon = jj; break; }
+    }
+  }
+  if (lane == 0) canon_out[i] = canon;
+}
+
+// ---- compaction ----------------------------------------------------------------------------------------------
+// One block: rank[i] = number of unique paths with a smaller index; also clears the multiplicities.
+__global__ void rank_kernel(const int32_t* __restrict__ canon, int n, int32_t* __restrict__ rank,
+                            int32_t* __restrict__ multiplicity, int32_t* __restrict__ num_unique) {
+  __shared__ int warp_tot[32];
+  __shared__ int carry_s;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  if (threadIdx.x == 0) carry_s = 0;
+  __syncthreads();
+  for (int base = 0; base < n; base += blockDim.x) {
+    const int i = base + threadIdx.x;
+    const int v = (i < n && canon[i] == i) ? 1 : 0;
+    if (i < n) multiplicity[i] = 0;
+    const uint32_t bal = __ballot_sync(0xffffffffu, v);
+    const int incl_w = __popc(bal & (0xffffffffu >> (31 - lane)));
+    if (lane == 31) warp_tot[warp] = incl_w;
+    __syncthreads();
+    if (warp == 0) {
+      int t = lane < nw ? warp_tot[lane] : 0;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int y = __shfl_up_sync(0xffffffffu, t, o);
+        if (lane >= o) t += y;
+      }
+      warp_tot[lane] = t;
+    }
+    __syncthreads();
+    const int before = carry_s + (warp ? warp_tot[warp - 1] : 0) + incl_w - v;
+    if (i < n) rank[i] = before;
+    __syncthreads();
+    if (threadIdx.x == blockDim.x - 1) carry_s = before + v;
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) *num_unique = carry_s;
+}
+
+__global__ void finalize_kernel(const int32_t* __restrict__ canon, const int32_t* __restrict__ rank, int n,
+                                const int32_t* __restrict__ slot_in, int32_t* __restrict__ path_to_unique,
+                                int32_t* __restrict__ unique_paths, int32_t* __restrict__ multiplicity,
+                                int32_t* __restrict__ slot_out) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const int c = canon[i];
+  const int r = rank[c];
+  path_to_unique[i] = r;
+  if (c == i) unique_paths[r] = i;
+  atomicAdd(&multiplicity[r], 1);
+  if (slot_out) slot_out[i] = slot_in[c];
+}
+
+__global__ void zero_scalar_kernel(int32_t* p) { *p = 0; }
+
+struct Layout {
+  size_t hash64, keys_a, keys_b, idx_a, idx_b, hist, rank, total;
+  int num_tiles;
+};
+
+static Layout layout(int n) {
+  Layout L;
+  const size_t m = n > 0 ? n : 1;
+  L.num_tiles = static_cast<int>((m + kSortTile - 1) / kSortTile);
+  size_t off = 0;
+  L.hash64 = off; off = align_up(off + m * 8);
+  L.keys_a = off; off = align_up(off + m * 4);
+  L.keys_b = off; off = align_up(off + m * 4);
+  L.idx_a = off; off = align_up(off + m * 4);
+  L.idx_b = off; off = align_up(off + m * 4);
+  L.hist = off; off = align_up(off + static_cast<size_t>(256) * L.num_tiles * 4);
+  L.rank = off; off = align_up(off + m * 4);
+  L.total = off;
+  return L;
+}
+
+}  // namespace dedup
+}  // namespace ss
+
+extern "C" int32_t ss_dedup_workspace_bytes(int32_t n_paths, size_t* out_bytes) {
+  if (n_paths < 0 || !out_bytes) return SS_ERR_INVALID_ARG;
+  *out_bytes = ss::dedup::layout(n_paths).total;
+  return SS_OK;
+}
+
+extern "C" int32_t ss_dedup_paths(const int32_t* tok_ids, const int64_t* tok_offsets, const int64_t* ctx_key,
+                                  const int32_t* slot_in, int32_t n_paths, uint32_t flags, int32_t* canon_out,
+                                  int32_t* path_to_unique_out, int32_t* unique_paths_out,
+                                  int32_t* multiplicity_out, int32_t* slot_out, int32_t* num_unique_out,
+                                  void* workspace, size_t workspace_bytes, void* stream) {
+  using namespace ss;
+  using namespace ss::dedup;
+  if (n_paths < 0 || !num_unique_out) return SS_ERR_INVALID_ARG;
+  if ((slot_in == nullptr) != (slot_out == nullptr)) return SS_ERR_INVALID_ARG;
+  if (flags & ~SS_FLAG_WEAK_HASH) return SS_ERR_INVALID_ARG;
+  cudaStream_t st = as_stream(stream);
+  if (n_paths == 0) {
+    SS_LAUNCH(zero_scalar_kernel, 1, 1, 0, st, num_unique_out);
+    return SS_OK;
+  }
+  if (!tok_offsets || !canon_out || !path_to_unique_out || !unique_paths_out || !multiplicity_out || !workspace)
+    return SS_ERR_INVALID_ARG;
+  if (!tok_ids) return SS_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return SS_ERR_INVALID_ARG;
+  const Layout L = layout(n_paths);
+  if (workspace_bytes < L.total) return SS_ERR_WORKSPACE_TOO_SMALL;
+  char* ws = static_cast<char*>(workspace);
+  uint64_t* hash64 = reinterpret_cast<uint64_t*>(ws + L.hash64);
+  uint32_t* keys_a = reinterpret_cast<uint32_t*>(ws + L.keys_a);
+  uint32_t* keys_b = reinterpret_cast<uint32_t*>(ws + L.keys_b);
+  uint32_t* idx_a = reinterpret_cast<uint32_t*>(ws + L.idx_a);
+  uint32_t* idx_b = reinterpret_cast<uint32_t*>(ws + L.idx_b);
+  uint32_t* hist = reinterpret_cast<uint32_t*>(ws + L.hist);
+  int32_t* rank = reinterpret_cast<int32_t*>(ws + L.rank);
+
+  const int n = n_paths;
+  const uint32_t weak = (flags & SS_FLAG_WEAK_HASH) ? 1u : 0u;
+  const int warps_per_block = 8;
+  const int warp_blocks = (n + warps_per_block - 1) / warps_per_block;
+  SS_LAUNCH(hash_kernel, warp_blocks, warps_per_block * 32, 0, st, tok_ids, tok_offsets, ctx_key, n, weak, hash64,
+            keys_a, idx_a);
+  const int passes = weak ? 1 : 4;
+  uint32_t *kin = keys_a, *kout = keys_b, *iin = idx_a, *iout = idx_b;
+  for (int p = 0; p < passes; ++p) {
+    const int shift = 8 * p;
+    SS_LAUNCH(rs_hist, L.num_tiles, kSortThreads, 0, st, kin, n, shift, L.num_tiles, hist);
+    SS_LAUNCH(scan_u32_single_block, 1, 1024, 0, st, hist, 256 * L.num_tiles);
+    SS_LAUNCH(rs_scatter, L.num_tiles, kSortThreads, 0, st, kin, iin, kout, iout, n, shift, L.num_tiles, hist);
+    uint32_t* t = kin; kin = kout; kout = t;
+    t = iin; iin = iout; iout = t;
+  }
+  SS_LAUNCH(match_kernel, warp_blocks, warps_per_block * 32, 0, st, kin, iin, n, hash64, tok_ids, tok_offsets,
+            ctx_key, canon_out);
+  SS_LAUNCH(rank_kernel, 1, 1024, 0, st, canon_out, n, rank, multiplicity_out, num_unique_out);
+  SS_LAUNCH(finalize_kernel, (n + 255) / 256, 256, 0, st, canon_out, rank, n, slot_in, path_to_unique_out,
+            unique_paths_out, multiplicity_out, slot_out);
+  return SS_OK;
+}

@@ -1,0 +1,154 @@
+"""Device-side plumbing around the three C-ABI calls: uploads a synthetic workload, owns the output and
+workspace tensors, and runs   ss_dedup_paths -> (gather of the unique paths) -> ss_tree_attention -> ss_topk_prune.
+
+Only memory management and argument marshalling happen here.  The one data movement that is not a library call is
+the compaction of the per-path descriptor arrays and query rows by `unique_paths` - a plain gather that belongs
+to the caller (after deduplication a sequence has a single query row, so Q exists only for unique paths).
+"""
+from __future__ import annotations
+
+from typing import Dict, Optional
+
+import numpy as np
+import torch
+
+from . import binding as B
+from .synth import TreeWorkload
+
+
+def _dev(a: np.ndarray, device, dtype=None) -> torch.Tensor:
+    t = torch.from_numpy(np.ascontiguousarray(a))
+    if dtype is not None:
+        t = t.to(dtype)
+    return t.to(device)
+
+
+class DevicePipeline:
+    """Holds one workload on the GPU together with every buffer the three calls need (no allocation per step)."""
+
+    def __init__(self, w: TreeWorkload, device="cuda:0", attn_flags: int = 0, dedup_flags: int = 0,
+                 sm_scale: float = 0.0):
+        self.w = w
+        self.device = torch.device(device)
+        dev = self.device
+        self.attn_flags, self.dedup_flags, self.sm_scale = attn_flags, dedup_flags, sm_scale
+        N = w.num_paths
+        self.N = N
+        # ---- resident state: tree + KV pool ------------------------------------------------------------------
+        self.kv_pool = w.kv_pool.to(dev) if w.kv_pool.device != dev else w.kv_pool
+        self.node_parent = _dev(w.node_parent, dev)
+        self.node_kv_len = _dev(w.node_kv_len, dev)
+        self.node_page_offsets = _dev(w.node_page_offsets, dev)
+        self.node_pages = _dev(w.node_pages if w.node_pages.size else np.zeros(1, np.int32), dev)
+        # ---- per-step inputs (logical candidates) ----------------------------------------------------------
+        self.tok_ids = _dev(w.tok_ids if w.tok_ids.size else np.zeros(1, np.int32), dev)
+        self.tok_offsets = _dev(w.tok_offsets, dev)
+        self.ctx_key = _dev(w.ctx_key, dev)
+        self.slot_in = _dev(w.slot_in, dev)
+        self.path_leaf_node = _dev(w.path_leaf_node, dev)
+        self.path_q_len = _dev(w.path_q_len, dev)
+        self.q_offsets = _dev(w.q_offsets, dev)
+        self.q = w.q.to(dev) if w.q.device != dev else w.q
+        self.scores = _dev(w.scores, dev)
+        self.seg_offsets = _dev(w.seg_offsets, dev)
+        # ---- dedup outputs ----------------------------------------------------------------------------------------
+        i32 = dict(dtype=torch.int32, device=dev)
+        self.canon = torch.empty(max(N, 1), **i32)
+        self.path_to_unique = torch.empty(max(N, 1), **i32)
+        self.unique_paths = torch.empty(max(N, 1), **i32)
+        self.multiplicity = torch.empty(max(N, 1), **i32)
+        self.slot_out = torch.empty(max(N, 1), **i32)
+        self.num_unique = torch.zeros(1, **i32)
+        self.dedup_ws = B.alloc_workspace(B.ss_dedup_workspace_bytes(N), dev)
+        # ---- compacted (unique-path) descriptor arrays; capacity N ---------------------------------------------
+        self.u_leaf = torch.empty(max(N, 1), **i32)
+        self.u_q_len = torch.empty(max(N, 1), **i32)
+        self.u_q_offsets = torch.zeros(N + 1, dtype=torch.int64, device=dev)
+        total_q = w.total_q
+        self.u_q = torch.empty((max(total_q, 1), w.num_q_heads, w.head_dim), dtype=torch.bfloat16, device=dev)
+        self.out = torch.empty_like(self.u_q)
+        self.lse = torch.empty((max(total_q, 1), w.num_q_heads), dtype=torch.float32, device=dev)
+        self.q_row_of = torch.empty(max(total_q, 1), dtype=torch.int64, device=dev)
+        depth = self._max_depth(w)
+        self.desc = B.make_attn_desc(
+            num_q_heads=w.num_q_heads, num_kv_heads=w.num_kv_heads, kv_pool=self.kv_pool,
+            node_parent=self.node_parent, node_kv_len=self.node_kv_len, node_page_offsets=self.node_page_offsets,
+            node_pages=self.node_pages, total_node_pages=int(w.node_page_offsets[-1]),
+            path_leaf_node=self.u_leaf, path_q_len=self.u_q_len, q_offsets=self.u_q_offsets, total_q=total_q,
+            q=self.u_q, out=self.out, lse=self.lse, num_paths=N, num_paths_dev=self.num_unique,
+            sm_scale=sm_scale, flags=attn_flags, max_depth=depth,
+            max_decode_paths=int((w.path_q_len == 1).sum()))
+        self.attn_ws = B.alloc_workspace(B.ss_tree_attention_workspace_bytes(self.desc), dev)
+        # ---- top-k -----------------------------------------------------------------------------------------------
+        self.P = int(w.seg_offsets.shape[0]) - 1
+        self.survivors = torch.empty((max(self.P, 1), w.top_k), **i32)
+        self.keep = torch.empty(max(N, 1), dtype=torch.uint8, device=dev)
+        self.topk_ws = B.alloc_workspace(B.ss_topk_workspace_bytes(N), dev)
+
+    @staticmethod
+    def _max_depth(w: TreeWorkload) -> int:
+        depth = np.zeros(w.num_nodes, np.int32)
+        for n in range(w.num_nodes):          # parents come first
+            p = int(w.node_parent[n])
+            depth[n] = 1 if p < 0 else depth[p] + 1
+        return int(depth.max()) if w.num_nodes else 1
+
+    # ------------------------------------------------------------------------------------------------------------
+    def dedup(self, stream=None):
+        B.ss_dedup_paths(self.tok_ids, self.tok_offsets, self.ctx_key, self.slot_in, self.N, self.dedup_flags,
+                         self.canon, self.path_to_unique, self.unique_paths, self.multiplicity, self.slot_out,
+                         self.num_unique, self.dedup_ws, stream=stream)
+
+    def compact_unique(self):
+        """Gather of the unique paths' descriptor rows and query rows (device-side, no host sync: entries past
+        the live count U are computed from clamped indices and ignored by the attention call)."""
+        N = self.N
+        if N == 0:
+            return
+        U = self.num_unique
+        ar = torch.arange(N, device=self.device)
+        live = ar < U
+        src = torch.where(live, self.unique_paths[:N].long(), torch.zeros_like(ar))
+        self.u_leaf[:N] = self.path_leaf_node[src]
+        T = torch.where(live, self.path_q_len[src].long(), torch.zeros_like(ar))
+        self.u_q_len[:N] = T.to(torch.int32)
+        self.u_q_offsets[1:] = torch.cumsum(T, 0)
+        # query rows: row r of the compacted Q comes from row q_offsets[src[p]] + (r - u_q_offsets[p])
+        total = self.w.total_q
+        if total:
+            rows = torch.arange(total, device=self.device)
+            p = torch.searchsorted(self.u_q_offsets[1:], rows, right=True).clamp_(max=N - 1)
+            src_row = self.q_offsets[src[p]] + (rows - self.u_q_offsets[p])
+            src_row.clamp_(0, total - 1)
+            self.q_row_of[:total] = src_row
+            torch.index_select(self.q, 0, src_row, out=self.u_q[:total])
+
+    def attention(self, stream=None):
+        B.ss_tree_attention(self.desc, self.attn_ws, stream=stream)
+
+    def topk(self, stream=None):
+        B.ss_topk_prune(self.scores, self.seg_offsets, self.P, self.N, self.w.top_k, self.survivors, self.keep,
+                        self.topk_ws, stream=stream)
+
+    def step(self):
+        """One pass of the whole hot path."""
+        self.dedup()
+        self.compact_unique()
+        self.attention()
+        self.topk()
+
+    # ------------------------------------------------------------------------------------------------------------
+    def results(self) -> Dict[str, np.ndarray]:
+        torch.cuda.synchronize(self.device)
+        st = B.ss_last_device_status(self.attn_ws)
+        if st != B.SS_OK:
+            raise B.SpecScaleError(st, "ss_tree_attention (device status)")
+        U = int(self.num_unique.item())
+        N = self.N
+        tq = int(self.u_q_offsets[U].item()) if N else 0
+        return dict(
+            num_unique=U, canon=self.canon[:N].cpu().numpy(), path_to_unique=self.path_to_unique[:N].cpu().numpy(),
+            unique_paths=self.unique_paths[:U].cpu().numpy(), multiplicity=self.multiplicity[:U].cpu().numpy(),
+            slot_out=self.slot_out[:N].cpu().numpy(), total_q=tq,
+            out=self.out[:tq].to(torch.float64).cpu().numpy(), lse=self.lse[:tq].to(torch.float64).cpu().numpy(),
+            survivors=self.survivors[:self.P].cpu().numpy(), keep=self.keep[:N].cpu().numpy())

@@ -1,0 +1,382 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same seeded inputs.
+
+Bars (BASELINE the benchmark spec): dedup / remap / top-k bit-exact; attention |out - oracle| <= 2e-2 max and <= 2e-3
+mean, |lse - oracle| <= 1e-3.  Tighter internal gates (4e-3 max, 3e-4 mean, 1e-4 lse... see TIGHT below) catch
+indexing slips that the official bars would let through on long paths.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2609_39334_b200 import binding as B
+from paper_2609_39334_b200 import synth
+from paper_2609_39334_b200.pipeline import DevicePipeline
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+OUT_MAX, OUT_MEAN, LSE_MAX = 2e-2, 2e-3, 1e-3          # official
+TIGHT_OUT_MAX, TIGHT_OUT_MEAN, TIGHT_LSE = 6e-3, 4e-4, 2e-4   # internal, random N(0,1) data
+
+
+def check_dedup(r, w):
+    ref = oracle.dedup(w.tok_ids, w.tok_offsets, w.ctx_key, w.slot_in)
+    assert r["num_unique"] == ref["num_unique"]
+    for key in ("canon", "path_to_unique", "unique_paths", "multiplicity", "slot_out"):
+        assert np.array_equal(r[key], ref[key]), key
+    return ref
+
+
+def check_topk(r, w):
+    s_ref, k_ref = oracle.topk(w.scores, w.seg_offsets, w.top_k)
+    assert np.array_equal(r["survivors"], s_ref)
+    assert np.array_equal(r["keep"], k_ref)
+
+
+def sample_unique(ref, w, max_paths, seed=0):
+    """Indices INTO the unique list: all if few, else a seeded sample that contains the extremes."""
+    U = ref["num_unique"]
+    if U <= max_paths:
+        return np.arange(U)
+    uniq = ref["unique_paths"]
+    lens = np.asarray([w.node_kv_len[w.path_leaf_node[u]] for u in uniq])
+    T = w.path_q_len[uniq]
+    must = {0, U - 1, int(lens.argmin()), int(lens.argmax()), int(T.argmax()), int(T.argmin())}
+    mult = ref["multiplicity"]
+    if (mult > 1).any():
+        must.add(int(np.nonzero(mult > 1)[0][0]))
+    rng = np.random.default_rng(seed)
+    rest = rng.choice(U, size=max_paths - len(must), replace=False)
+    return np.asarray(sorted(must | set(int(x) for x in rest)))[:max_paths]
+
+
+def check_attention(r, w, ref, max_paths=48, tight=True, host_w=None):
+    """Compares the GPU rows of a sample of unique paths with the oracle."""
+    sel = sample_unique(ref, w, max_paths)
+    uniq = ref["unique_paths"][sel]
+    src = host_w if host_w is not None else w
+    o_ref, l_ref = oracle.tree_attention_workload(src, paths=uniq)
+    # rows of the selected unique paths in the compacted GPU output
+    T_u = w.path_q_len[ref["unique_paths"]].astype(np.int64)
+    off = np.concatenate([[0], np.cumsum(T_u)])
+    rows = np.concatenate([np.arange(off[i], off[i + 1]) for i in sel])
+    out, lse = r["out"][rows], r["lse"][rows]
+    assert np.isfinite(out).all(), "NaN/inf in attention output (poisoned slot read?)"
+    err = np.abs(out - o_ref)
+    fin = np.isfinite(l_ref)
+    assert np.array_equal(np.isfinite(lse), fin)
+    lerr = np.abs(lse[fin] - l_ref[fin]).max() if fin.any() else 0.0
+    assert err.max() <= OUT_MAX and err.mean() <= OUT_MEAN and lerr <= LSE_MAX, (err.max(), err.mean(), lerr)
+    if tight:
+        assert err.max() <= TIGHT_OUT_MAX and err.mean() <= TIGHT_OUT_MEAN and lerr <= TIGHT_LSE, \
+            (err.max(), err.mean(), lerr)
+    return err.max(), err.mean(), lerr
+
+
+MODES = [("fast", 0), ("no_tcgen05", B.SS_FLAG_NO_TCGEN05), ("generic", B.SS_FLAG_FORCE_GENERIC)]
+
+
+# =========================================================================================================
+# whole pipeline on the benchmark configurations
+# =========================================================================================================
+@pytest.mark.parametrize("mode,flags", MODES)
+@pytest.mark.parametrize("cfg", [1, 2, 3, 4])
+def test_pipeline_configs(cfg, mode, flags):
+    if mode == "generic" and cfg in (3,):
+        scale = 0.25
+    else:
+        scale = 1.0
+    w = synth.make_config(cfg, scale=scale)
+    pipe = DevicePipeline(w, DEV, attn_flags=flags | B.SS_FLAG_VALIDATE)
+    pipe.step()
+    r = pipe.results()
+    ref = check_dedup(r, w)
+    check_topk(r, w)
+    check_attention(r, w, ref, max_paths=40 if cfg != 3 else 12)
+    # duplicates read their result through path_to_unique: identical by construction
+    assert r["num_unique"] <= w.num_paths
+
+
+def test_pipeline_config1_all_rows_and_fullseq_dedup():
+    w = synth.make_config(1)
+    pipe = DevicePipeline(w, DEV)
+    pipe.step()
+    r = pipe.results()
+    ref = check_dedup(r, w)
+    check_attention(r, w, ref, max_paths=8)
+    # config 1 also de-duplicates on the full prefix+suffix token sequence with a null context
+    rng = np.random.default_rng(1)
+    prefix = rng.integers(0, synth.VOCAB, size=256).astype(np.int32)
+    seqs = [np.concatenate([prefix, w.tok_ids[w.tok_offsets[i]:w.tok_offsets[i + 1]]]) for i in range(8)]
+    ids = np.concatenate(seqs).astype(np.int32)
+    off = np.concatenate([[0], np.cumsum([len(s) for s in seqs])]).astype(np.int64)
+    got = run_dedup(ids, off, None, None)
+    want = oracle.dedup(ids, off)
+    for key in ("canon", "path_to_unique", "unique_paths", "multiplicity"):
+        assert np.array_equal(got[key], want[key])
+
+
+# =========================================================================================================
+# dedup
+# =========================================================================================================
+def run_dedup(ids, off, ctx, slot, flags=0):
+    n = len(off) - 1
+    dev = torch.device(DEV)
+    t = lambda a, dt: None if a is None else torch.from_numpy(np.ascontiguousarray(a, dtype=dt)).to(dev)
+    ids_t = t(ids if len(ids) else np.zeros(1, np.int32), np.int32)
+    i32 = dict(dtype=torch.int32, device=dev)
+    m = max(n, 1)
+    canon, p2u, uniq, mult = (torch.full((m,), -7, **i32) for _ in range(4))
+    slot_out = torch.full((m,), -7, **i32) if slot is not None else None
+    nu = torch.full((1,), -7, **i32)
+    ws = B.alloc_workspace(B.ss_dedup_workspace_bytes(n), dev)
+    B.ss_dedup_paths(ids_t, t(off, np.int64), t(ctx, np.int64), t(slot, np.int32), n, flags, canon, p2u, uniq, mult,
+                     slot_out, nu, ws)
+    torch.cuda.synchronize()
+    U = int(nu.item())
+    return dict(num_unique=U, canon=canon[:n].cpu().numpy(), path_to_unique=p2u[:n].cpu().numpy(),
+                unique_paths=uniq[:U].cpu().numpy(), multiplicity=mult[:U].cpu().numpy(),
+                slot_out=None if slot is None else slot_out[:n].cpu().numpy())
+
+
+def dedup_case(rng, n, alphabet, max_len, n_ctx):
+    lens = rng.integers(0, max_len + 1, size=n)
+    off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    ids = rng.integers(0, alphabet, size=int(off[-1])).astype(np.int32)
+    ctx = rng.integers(0, n_ctx, size=n).astype(np.int64)
+    slot = rng.integers(0, 1 << 20, size=n).astype(np.int32)
+    return ids, off, ctx, slot
+
+
+@pytest.mark.parametrize("flags", [0, B.SS_FLAG_WEAK_HASH])
+@pytest.mark.parametrize("n,alphabet,max_len,n_ctx", [
+    (1, 3, 4, 1), (2, 2, 2, 1), (37, 2, 3, 2), (300, 3, 5, 2), (2049, 4, 6, 3), (5000, 2, 40, 1), (20000, 50, 3, 4),
+])
+def test_dedup_random_collision_heavy(n, alphabet, max_len, n_ctx, flags):
+    rng = np.random.default_rng(n * 31 + alphabet)
+    ids, off, ctx, slot = dedup_case(rng, n, alphabet, max_len, n_ctx)
+    got = run_dedup(ids, off, ctx, slot, flags)
+    want = oracle.dedup(ids, off, ctx, slot)
+    assert got["num_unique"] == want["num_unique"]
+    for key in ("canon", "path_to_unique", "unique_paths", "multiplicity", "slot_out"):
+        assert np.array_equal(got[key], want[key]), key
+
+
+def test_dedup_edge_cases():
+    got = run_dedup(np.zeros(0, np.int32), np.zeros(1, np.int64), None, None)
+    assert got["num_unique"] == 0
+    # all empty sequences, null ctx: one class
+    got = run_dedup(np.zeros(0, np.int32), np.zeros(6, np.int64), None, None)
+    assert got["num_unique"] == 1 and list(got["canon"]) == [0] * 5 and list(got["multiplicity"]) == [5]
+    # all identical long sequences
+    seq = np.arange(1000, dtype=np.int32)
+    ids = np.tile(seq, 64)
+    off = (np.arange(65) * 1000).astype(np.int64)
+    got = run_dedup(ids, off, None, np.arange(64, dtype=np.int32))
+    assert got["num_unique"] == 1 and list(got["slot_out"]) == [0] * 64
+    # differ only in the last token / only in length / only in ctx
+    ids = np.asarray([1, 2, 3, 1, 2, 4, 1, 2, 1, 2, 3], np.int32)
+    off = np.asarray([0, 3, 6, 8, 11], np.int64)
+    got = run_dedup(ids, off, np.asarray([0, 0, 0, 1], np.int64), None)
+    assert list(got["canon"]) == [0, 1, 2, 3]
+    got = run_dedup(ids, off, np.asarray([5, 5, 5, 5], np.int64), None)
+    assert list(got["canon"]) == [0, 1, 2, 0]
+    # tok_offsets that do not start at zero
+    got = run_dedup(np.asarray([9, 9, 7, 7, 7, 7], np.int32), np.asarray([2, 4, 6], np.int64), None, None)
+    assert list(got["canon"]) == [0, 0]
+
+
+def test_dedup_paper_example_on_gpu():
+    got = run_dedup(np.asarray([1055, 1055, 1055, 429], np.int32), np.arange(5, dtype=np.int64), np.zeros(4, np.int64), None)
+    assert list(got["multiplicity"]) == [3, 1]
+
+
+def test_dedup_idempotent_and_permutation_invariant_on_gpu():
+    rng = np.random.default_rng(77)
+    ids, off, ctx, slot = dedup_case(rng, 4000, 3, 4, 2)
+    r = run_dedup(ids, off, ctx, None)
+    seqs = [ids[off[i]:off[i + 1]] for i in range(4000)]
+    u = r["unique_paths"]
+    ids2 = np.concatenate([seqs[i] for i in u]).astype(np.int32)
+    off2 = np.concatenate([[0], np.cumsum([len(seqs[i]) for i in u])]).astype(np.int64)
+    r2 = run_dedup(ids2, off2, ctx[u], None)
+    assert r2["num_unique"] == len(u) and np.array_equal(r2["canon"], np.arange(len(u)))
+    perm = rng.permutation(4000)
+    ids3 = np.concatenate([seqs[i] for i in perm]).astype(np.int32) if len(ids) else ids
+    off3 = np.concatenate([[0], np.cumsum([len(seqs[i]) for i in perm])]).astype(np.int64)
+    r3 = run_dedup(ids3, off3, ctx[perm], None)
+    assert r3["num_unique"] == r["num_unique"]
+    inv = np.argsort(perm)
+    cls_min = {}
+    for i in range(4000):
+        c = int(r["canon"][i])
+        cls_min[c] = min(cls_min.get(c, 1 << 30), int(inv[i]))
+    assert all(int(r3["canon"][inv[i]]) == cls_min[int(r["canon"][i])] for i in range(4000))
+
+
+# =========================================================================================================
+# top-k
+# =========================================================================================================
+def run_topk(scores, seg, k):
+    dev = torch.device(DEV)
+    n, P = len(scores), len(seg) - 1
+    sc = torch.from_numpy(np.ascontiguousarray(scores if n else np.zeros(1, np.float32), dtype=np.float32)).to(dev)
+    sg = torch.from_numpy(np.ascontiguousarray(seg, dtype=np.int32)).to(dev)
+    surv = torch.full((max(P, 1), k), -9, dtype=torch.int32, device=dev)
+    keep = torch.full((max(n, 1),), 7, dtype=torch.uint8, device=dev)
+    ws = B.alloc_workspace(B.ss_topk_workspace_bytes(n), dev)
+    B.ss_topk_prune(sc, sg, P, n, k, surv, keep, ws)
+    torch.cuda.synchronize()
+    return surv[:P].cpu().numpy(), keep[:n].cpu().numpy()
+
+
+@pytest.mark.parametrize("sizes,k", [
+    ([32] * 8, 8), ([0, 5, 0, 1, 70], 4), ([4096], 64), ([5000, 3, 9000], 100), ([20000], 1), ([7], 16), ([256] * 64, 64),
+])
+def test_topk_vs_oracle(sizes, k):
+    rng = np.random.default_rng(sum(sizes) + k)
+    seg = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int32)
+    n = int(seg[-1])
+    for variant in range(2):
+        if variant == 0:
+            sc = rng.random(n).astype(np.float32)
+        else:                                   # tie-heavy, large mass at the perfect score
+            sc = (rng.integers(0, 9, size=n) / 8.0).astype(np.float32)
+            sc[rng.random(n) < 0.3] = 1.0
+        surv, keep = run_topk(sc, seg, k)
+        s_ref, k_ref = oracle.topk(sc, seg, k)
+        assert np.array_equal(surv, s_ref) and np.array_equal(keep, k_ref)
+
+
+def test_topk_special_values_and_gaps():
+    sc = np.asarray([0.0, -0.0, np.nan, 0.5, np.nan, -1.0, np.inf, -np.inf, 3.0, 3.0], np.float32)
+    surv, keep = run_topk(sc, [0, 8], 8)          # candidates 8, 9 belong to no segment
+    assert list(surv[0]) == [6, 3, 0, 1, 5, 7, 2, 4] and list(keep[8:]) == [0, 0]
+    s_ref, k_ref = oracle.topk(sc, [0, 8], 3)
+    surv, keep = run_topk(sc, [0, 8], 3)
+    assert np.array_equal(surv, s_ref) and np.array_equal(keep[:8], k_ref[:8])
+
+
+def test_topk_beam_bookkeeping_on_gpu():
+    rng = np.random.default_rng(3)
+    for N, M in [(4, 4), (8, 4), (16, 4), (32, 4)]:
+        sc = rng.random(N).astype(np.float32)
+        surv, keep = run_topk(sc, [0, N], N // M)
+        assert int(keep.sum()) == N // M and set(surv[0]) == set(np.argsort(-sc, kind="stable")[:N // M])
+
+
+# =========================================================================================================
+# attention: shapes beyond the configs, closed forms, invariances
+# =========================================================================================================
+def attention_only(w, flags=0, sm_scale=0.0):
+    pipe = DevicePipeline(w, DEV, attn_flags=flags | B.SS_FLAG_VALIDATE, sm_scale=sm_scale)
+    pipe.dedup()
+    pipe.compact_unique()
+    pipe.attention()
+    r = pipe.results()
+    ref = oracle.dedup(w.tok_ids, w.tok_offsets, w.ctx_key, w.slot_in)
+    return r, ref
+
+
+SHAPES = [
+    # name, Hq, Hkv, levels, fanout, problems, leaf range, T-fn, dup
+    ("gqa1_deep", 4, 4, [64, 32, 16], [2, 3, 2], 2, (0, 70), lambda i, n, rng: 1, 0.2),
+    ("gqa7_mixed", 28, 4, [192], [9], 3, (0, 150), lambda i, n, rng: 1 if i % 3 else int(rng.integers(2, 50)), 0.1),
+    ("gqa8_verify_ragged", 16, 2, [128, 64], [2, 5], 2, (1, 200), lambda i, n, rng: int(rng.integers(16, 129)), 0.0),
+    ("gqa16_decode", 32, 2, [256], [40], 2, (0, 300), lambda i, n, rng: 1, 0.3),
+    ("gqa2_small_T", 8, 4, [48], [6], 2, (3, 40), lambda i, n, rng: int(rng.integers(1, 6)), 0.0),
+    ("gqa32_generic_decode", 32, 1, [64], [5], 1, (1, 90), lambda i, n, rng: 1 + (i % 2) * 20, 0.0),
+    ("no_prefix", 12, 2, [0], [7], 2, (0, 130), lambda i, n, rng: 1 + (i % 2) * 17, 0.0),
+    ("long_prefix_few_paths", 8, 2, [4096], [3], 1, (5, 600), lambda i, n, rng: 1, 0.0),
+]
+
+
+@pytest.mark.parametrize("mode,flags", MODES)
+@pytest.mark.parametrize("shape", SHAPES, ids=[s[0] for s in SHAPES])
+def test_attention_shapes(shape, mode, flags):
+    name, Hq, Hkv, levels, fanout, problems, leaf, qfn, dup = shape
+    w = synth.build_tree_workload(name, 1234, Hq, Hkv, levels, fanout, problems, leaf, qfn, dup_frac=dup)
+    r, ref = attention_only(w, flags)
+    check_attention(r, w, ref, max_paths=64)
+
+
+@pytest.mark.parametrize("mode,flags", MODES)
+def test_attention_closed_forms(mode, flags):
+    """Q == 0 => lse = ln(visible), out = mean of the visible V rows; with V[j,:] = position j (< 256, exact in
+    bf16) that mean is (visible-1)/2.  Catches off-by-one in masks, page order and node lengths at tight
+    tolerance."""
+    for levels, fanout, T in [([64], [5], 1), ([32, 48], [2, 3], 1), ([80], [3], 24), ([64], [2], 3)]:
+        w = synth.build_tree_workload("cf", 99, 8, 2, levels, fanout, 1, (0, 100), lambda i, n, rng: T)
+        w.q.zero_()
+        for p in range(w.num_paths):
+            pos = 0
+            for n in w.chain(int(w.path_leaf_node[p])):
+                pages = w.node_pages[w.node_page_offsets[n]:w.node_page_offsets[n + 1]]
+                for j in range(int(w.node_kv_len[n])):
+                    w.kv_pool[int(pages[j // 16]), 1, :, j % 16, :] = float(pos)
+                    pos += 1
+            assert pos <= 256
+        r, ref = attention_only(w, flags)
+        row = 0
+        for u in ref["unique_paths"]:
+            L = w.path_kv_len(int(u))
+            for t in range(T):
+                vis = L - T + t + 1
+                if vis <= 0:
+                    assert np.all(r["out"][row] == 0) and np.all(np.isneginf(r["lse"][row]))
+                else:
+                    np.testing.assert_allclose(r["lse"][row], math.log(vis), atol=2e-5)
+                    # bf16 output rounding: relative 2^-9
+                    np.testing.assert_allclose(r["out"][row], (vis - 1) / 2.0, rtol=2.0 ** -8, atol=1e-6)
+                row += 1
+
+
+def test_attention_page_permutation_and_explicit_scale():
+    w = synth.build_tree_workload("perm", 5, 12, 2, [128], [6], 2, (1, 120), lambda i, n, rng: 1 + (i % 2) * 30)
+    r1, ref = attention_only(w, sm_scale=0.05)
+    o_ref, l_ref = oracle.tree_attention_workload(w, paths=ref["unique_paths"], sm_scale=0.05)
+    assert np.abs(r1["out"] - o_ref).max() <= TIGHT_OUT_MAX and np.abs(r1["lse"] - l_ref).max() <= TIGHT_LSE
+    rng = np.random.default_rng(0)
+    perm = rng.permutation(w.num_pages)
+    new_pool = torch.empty_like(w.kv_pool)
+    new_pool[torch.from_numpy(perm)] = w.kv_pool
+    w.kv_pool = new_pool
+    w.node_pages = perm[w.node_pages].astype(np.int32)
+    r2, _ = attention_only(w, sm_scale=0.05)
+    assert np.abs(r2["out"] - r1["out"]).max() <= 2 * TIGHT_OUT_MAX
+    assert np.abs(r2["lse"] - r1["lse"]).max() <= 2 * TIGHT_LSE
+
+
+def test_attention_empty_and_degenerate():
+    # every path empty: out = 0, lse = -inf
+    w = synth.build_tree_workload("empty", 3, 4, 2, [0], [3], 1, (0, 0), lambda i, n, rng: 1)
+    r, ref = attention_only(w)
+    assert np.all(r["out"] == 0) and np.all(np.isneginf(r["lse"]))
+    # no paths at all
+    w = synth.build_tree_workload("p0", 3, 4, 2, [16], [0], 1, (0, 0), lambda i, n, rng: 1)
+    pipe = DevicePipeline(w, DEV)
+    pipe.step()
+    assert pipe.results()["num_unique"] == 0
+
+
+def test_attention_device_errors_are_reported():
+    w = synth.build_tree_workload("bad", 3, 4, 2, [32], [3], 1, (1, 20), lambda i, n, rng: 1)
+    pipe = DevicePipeline(w, DEV, attn_flags=B.SS_FLAG_VALIDATE)
+    pipe.dedup()
+    pipe.compact_unique()
+    pipe.node_pages[0] = 10 ** 6                     # out-of-range page id: caught by the validator, never read
+    pipe.attention()
+    torch.cuda.synchronize()
+    assert B.ss_last_device_status(pipe.attn_ws) == B.SS_ERR_BAD_INPUT
+    pipe.node_pages[0] = int(w.node_pages[0])
+    pipe.attention()
+    torch.cuda.synchronize()
+    assert B.ss_last_device_status(pipe.attn_ws) == B.SS_OK
+    # a tree deeper than SS_MAX_DEPTH is refused, not walked
+    deep = synth.build_tree_workload("deep", 3, 4, 2, [16] * 17, [1] * 17, 1, (1, 5), lambda i, n, rng: 1)
+    pipe = DevicePipeline.__new__(DevicePipeline)
+    with pytest.raises(B.SpecScaleError):
+        DevicePipeline.__init__(pipe, deep, DEV)     # max_depth hint 18 > SS_MAX_DEPTH: rejected on the host
