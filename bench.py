@@ -1,0 +1,398 @@
+#!/usr/bin/env python
+"""Benchmark of the candidate-path hot path: one step = ss_dedup_paths -> gather of the unique paths ->
+ss_tree_attention -> ss_topk_prune over one batch of seeded synthetic candidate trees.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c3|c4|c5] [--impl reference]
+
+Prints ONE JSON line.  metric = candidate-path query tokens/s (query tokens of all N logical candidates divided
+by the step time).  `value` has every input resident in HBM; `e2e` copies the step's inputs from pinned host
+memory and reads the results back inside the timed region.  `roofline` is for the dominant attention kernel,
+timed live with CUDA events on the launching stream.  `cpu_baseline` is the CPU oracle on a bounded sample.
+With --impl reference the CPU oracle is the timed arm.  Under torchrun every rank runs its own replica of the
+workload (disjoint problems, no collective on the data path; weak scaling).
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "candidate_path_query_tokens_per_s"
+UNIT = "tokens/s"
+WORKLOADS = {"c2": 2, "c3": 3, "c4": 4, "c5": 5}
+L2_BYTES = 126 * 1024 * 1024
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_burst=float(p["bf16_tflops"]),
+                    bf16_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_burst=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+# ------------------------------------------------------------------------------------------------------------
+# algorithmic work of one step (what the method must do; computed from the tree and the unique set)
+# ------------------------------------------------------------------------------------------------------------
+def algorithmic_work(w, unique_paths):
+    """-> dict(tile_flops, leaf_bytes, unique_kv_bytes, tokens).  flops = 4*D per unmasked (query row, key) pair
+    of the rows that run on the tensor-core tiles (shared nodes of decode paths, whole chain of verification
+    paths); leaf bytes = K+V bytes of the private leaves of unique decode paths, read once."""
+    D, Hq, Hkv = w.head_dim, w.num_q_heads, w.num_kv_heads
+    kv_token_bytes = 2 * Hkv * D * 2
+    node_start = np.zeros(w.num_nodes, np.int64)
+    for n in range(w.num_nodes):
+        p = int(w.node_parent[n])
+        node_start[n] = 0 if p < 0 else node_start[p] + int(w.node_kv_len[p])
+    leaf = w.path_leaf_node[unique_paths]
+    T = w.path_q_len[unique_paths].astype(np.int64)
+    leaf_len = w.node_kv_len[leaf].astype(np.int64)
+    prefix_len = node_start[leaf]
+    L = prefix_len + leaf_len
+    dec = T == 1
+    pairs_dec_shared = int(prefix_len[dec].sum())
+    # verification: sum_t (L - T + t + 1) = T*L - T*(T-1)/2
+    Tv, Lv = T[~dec], L[~dec]
+    pairs_ver = int((Tv * Lv - Tv * (Tv - 1) // 2).sum())
+    tile_flops = 4.0 * D * Hq * (pairs_dec_shared + pairs_ver)
+    leaf_bytes = float(leaf_len[dec].sum()) * kv_token_bytes
+    used_nodes = np.zeros(w.num_nodes, bool)
+    for l in np.unique(leaf):
+        n = int(l)
+        while n >= 0 and not used_nodes[n]:
+            used_nodes[n] = True
+            n = int(w.node_parent[n])
+    unique_kv_bytes = float(w.node_kv_len[used_nodes].astype(np.int64).sum()) * kv_token_bytes
+    return dict(tile_flops=tile_flops, leaf_bytes=leaf_bytes, unique_kv_bytes=unique_kv_bytes,
+                tokens=int(w.path_q_len.astype(np.int64).sum()))
+
+
+# ------------------------------------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu_index = gpu_index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu_index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        self.proc.terminate()          # the exact process started above
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        sm, smax, reasons = [], [], set()
+        for r in self.rows:
+            if len(r) < 9:
+                continue
+            try:
+                sm.append(float(r[1]))
+                smax.append(float(r[2]))
+            except ValueError:
+                continue
+            for name, col in (("hw_slowdown", 5), ("hw_thermal_slowdown", 6), ("sw_thermal_slowdown", 7),
+                              ("sw_power_cap", 8)):
+                if r[col].lower() == "active":
+                    reasons.add(name)
+        return dict(sm_mhz=float(np.median(sm)) if sm else None, sm_max_mhz=max(smax) if smax else None,
+                    reasons=sorted(reasons), samples=len(sm))
+
+
+# ------------------------------------------------------------------------------------------------------------
+# CPU oracle arm (cpu_baseline leg and --impl reference)
+# ------------------------------------------------------------------------------------------------------------
+def oracle_sample(w, seed=0):
+    """A bounded sample of the workload for the CPU oracle: a few verification paths and more decode paths,
+    sized by the host core count for roughly 10-30 s of CPU work per pass."""
+    import oracle
+    cores = oracle.host_cores()
+    rng = np.random.default_rng(seed)
+    ded = oracle.dedup(w.tok_ids, w.tok_offsets, w.ctx_key, w.slot_in)
+    uniq = ded["unique_paths"]
+    T = w.path_q_len[uniq]
+    ver, dec = uniq[T > 1], uniq[T == 1]
+    # fp64 cost model: pairs * Hq * 2 * D multiply-adds; ~0.7 G mul-add/s per core for this plain loop
+    budget_pairs = 12.0 * cores * 0.7e9 / (2.0 * w.head_dim * w.num_q_heads)
+    chosen, pairs = [], 0.0
+    pools = [list(rng.permutation(ver)), list(rng.permutation(dec))]
+    while (pools[0] or pools[1]) and pairs < budget_pairs:
+        for pool in pools:
+            if pool:
+                p = int(pool.pop())
+                L = w.path_kv_len(p)
+                Tp = int(w.path_q_len[p])
+                pairs += Tp * L
+                chosen.append(p)
+    return np.asarray(sorted(chosen), np.int64)
+
+
+def time_oracle(w_host, sample, steps, warmup):
+    import oracle
+    times = []
+    for it in range(warmup + steps):
+        t0 = time.perf_counter()
+        oracle.dedup(w_host.tok_ids, w_host.tok_offsets, w_host.ctx_key, w_host.slot_in)
+        oracle.tree_attention_workload(w_host, paths=np.arange(w_host.num_paths))
+        oracle.topk(w_host.scores, w_host.seg_offsets, w_host.top_k)
+        if it >= warmup:
+            times.append(time.perf_counter() - t0)
+    return float(np.mean(times))
+
+
+# ------------------------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="c5", choices=sorted(WORKLOADS))
+    ap.add_argument("--scale", type=float, default=1.0, help="shrink the number of problems (debugging only)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    import torch
+    from paper_2609_39334_b200 import synth
+
+    cfg_idx = WORKLOADS[args.workload]
+
+    # ---------------------------------------------------------------------------------------------- reference arm
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        import oracle
+        oracle.build()
+        dev = "cuda:0" if torch.cuda.is_available() else "cpu"
+        w = synth.make_config(cfg_idx, device=dev, scale=args.scale)
+        sample = oracle_sample(w)
+        sub = synth.extract_subworkload(w, sample)
+        del w
+        if dev != "cpu":
+            torch.cuda.empty_cache()
+        sec = time_oracle(sub, sample, max(args.steps, 1), min(args.warmup, 1))
+        tokens = int(sub.path_q_len.astype(np.int64).sum())
+        val = tokens / sec
+        what = (f"{len(sample)} unique paths of {args.workload} ({int((sub.path_q_len > 1).sum())} verification, "
+                f"{int((sub.path_q_len == 1).sum())} decode), {tokens} query tokens per step")
+        print(json.dumps({
+            "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.workload, "sample": what},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": oracle.host_cores(), "kind": "oracle", "sample": what},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        }))
+        return
+
+    # ---------------------------------------------------------------------------------------------------- our arm
+    assert torch.cuda.is_available(), "bench.py needs a GPU (there is no CPU fallback)"
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    from paper_2609_39334_b200 import binding as B
+    from paper_2609_39334_b200.pipeline import DevicePipeline
+    B.lib()
+
+    # every rank its own problems: same shapes, different seed
+    w = synth.make_config(cfg_idx, device=dev, scale=args.scale, poison=True, replica=rank)
+    pipe = DevicePipeline(w, dev)
+    kv_bytes = pipe.kv_pool.numel() * 2
+    flush = None
+    if kv_bytes < 4 * L2_BYTES:
+        flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=dev)
+
+    def sync_all():
+        torch.cuda.synchronize(dev)
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize(dev)
+
+    # warm-up (also the functional check of the device status)
+    for _ in range(max(args.warmup, 1) if args.warmup else 0):
+        pipe.step()
+    torch.cuda.synchronize(dev)
+    if args.warmup:
+        st = B.ss_last_device_status(pipe.attn_ws)
+        if st != B.SS_OK:
+            raise B.SpecScaleError(st, "warm-up")
+
+    clocks = ClockSampler(local_rank)
+    if rank == 0:
+        clocks.start()
+        time.sleep(0.15)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    B.ss_profile_read()
+    B.ss_profile_enable(True)
+    launches0 = B.ss_launch_count()
+    sync_all()
+    for i in range(args.steps):
+        if flush is not None:
+            flush.fill_(i & 0xff)       # evicts the pool from L2 between iterations (outside the timed events)
+        ev[i][0].record()
+        pipe.step()
+        ev[i][1].record()
+    sync_all()
+    launches = B.ss_launch_count() - launches0
+    B.ss_profile_enable(False)
+    phase_ms, phase_calls = B.ss_profile_read()
+    clk = clocks.stop() if rank == 0 else None
+    step_ms = [a.elapsed_time(b) for a, b in ev]
+    total_ms = float(sum(step_ms))
+    if dist is not None:
+        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    st = B.ss_last_device_status(pipe.attn_ws)
+    if st != B.SS_OK:
+        raise B.SpecScaleError(st, "timed region")
+
+    U = int(pipe.num_unique.item())
+    unique_paths = pipe.unique_paths[:U].cpu().numpy()
+    work = algorithmic_work(w, unique_paths)
+    tokens = work["tokens"]
+    value = world * tokens / (ms_per_step * 1e-3)
+
+    # ---- roofline of the attention kernels (per launch, CUDA events on the launching stream) -----------------
+    peaks = load_peaks()
+    long_step = total_ms > 1000.0
+    tensor_peak = peaks["bf16_sustained"] if long_step else peaks["bf16_burst"]
+    traffic = {}
+    tpath = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    if os.path.exists(tpath):
+        with open(tpath) as f:
+            traffic = json.load(f).get(args.workload, {})
+    roofs = {}
+    if phase_calls["tiles"]:
+        t_ms = phase_ms["tiles"] / phase_calls["tiles"]
+        ach = work["tile_flops"] / (t_ms * 1e-3) / 1e12
+        roofs["tiles"] = {"kernel": "tile_items_umma_kernel", "bound": "tensor", "achieved": ach, "peak": tensor_peak,
+                          "unit": "TFLOP/s", "frac": ach / tensor_peak, "traffic": traffic.get("tiles"),
+                          "ms_per_launch": t_ms, "peak_kind": f"{peaks['source']} {'sustained' if long_step else 'burst'}"}
+    if phase_calls["leaves"]:
+        t_ms = phase_ms["leaves"] / phase_calls["leaves"]
+        ach = work["leaf_bytes"] / (t_ms * 1e-3) / 1e9
+        roofs["leaves"] = {"kernel": "leaf_items_kernel", "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"],
+                           "unit": "GB/s", "frac": ach / peaks["hbm_gbs"], "traffic": traffic.get("leaves"),
+                           "ms_per_launch": t_ms, "peak_kind": f"{peaks['source']} copy"}
+    dominant = max(roofs, key=lambda k: roofs[k]["ms_per_launch"]) if roofs else None
+    attn_ms = sum(phase_ms.values()) / max(phase_calls["plan"], 1)
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": args.workload, "paths": w.num_paths, "unique_paths": U, "query_tokens": tokens,
+                   "heads": f"{w.num_q_heads}q/{w.num_kv_heads}kv", "kv_pool_gb": kv_bytes / 1e9,
+                   "l2": "inputs larger than L2" if flush is None else "L2 flushed between iterations",
+                   "parallelism": f"replicas x{world}" if world > 1 else "single GPU"},
+        "gpu_launches": int(launches),
+        "attention_ms_per_step": attn_ms,
+        "attention_tokens_per_s": world * tokens / (attn_ms * 1e-3) if attn_ms > 0 else None,
+        "phase_ms_per_step": {k: (phase_ms[k] / phase_calls[k] if phase_calls[k] else 0.0) for k in phase_ms},
+        "roofline": roofs.get(dominant) if dominant else None,
+        "roofline_phases": roofs,
+        "unique_kv_gb": work["unique_kv_bytes"] / 1e9,
+        "clocks": clk,
+    }
+
+    # ---- end to end: inputs from pinned host memory, results back to the host, every step ---------------------
+    if not args.no_e2e:
+        h_in = {k: getattr(pipe, k) for k in ("tok_ids", "tok_offsets", "ctx_key", "slot_in", "path_leaf_node",
+                                               "path_q_len", "q_offsets", "q", "scores", "seg_offsets")}
+        pinned_in = {k: torch.empty(v.shape, dtype=v.dtype, pin_memory=True).copy_(v) for k, v in h_in.items()}
+        d_out = {k: getattr(pipe, k) for k in ("canon", "path_to_unique", "unique_paths", "multiplicity", "slot_out",
+                                                "num_unique", "out", "lse", "survivors", "keep")}
+        pinned_out = {k: torch.empty(v.shape, dtype=v.dtype, pin_memory=True) for k, v in d_out.items()}
+        h2d = sum(v.numel() * v.element_size() for v in pinned_in.values())
+        d2h = sum(v.numel() * v.element_size() for v in pinned_out.values())
+
+        def e2e_step():
+            for k, v in pinned_in.items():
+                h_in[k].copy_(v, non_blocking=True)
+            pipe.step()
+            for k, v in d_out.items():
+                pinned_out[k].copy_(v, non_blocking=True)
+
+        e2e_step()
+        sync_all()
+        n_e2e = max(3, min(args.steps, 5))
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(n_e2e):
+            e2e_step()
+        e1.record()
+        sync_all()
+        e2e_ms = e0.elapsed_time(e1) / n_e2e
+        if dist is not None:
+            t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = float(t.item())
+        out["e2e"] = {"value": world * tokens / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+                      "d2h_bytes_per_step": int(d2h), "ms_per_step": e2e_ms, "steps": n_e2e,
+                      "note": "KV pool stays resident (it is the cache); candidates, queries and scores come from "
+                              "pinned host memory, all results go back"}
+        del pinned_in, pinned_out
+
+    # ---- CPU oracle beside it (rank 0, N = 1 only) ----------------------------------------------------------------
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        oracle.build()
+        sample = oracle_sample(w)
+        sub = synth.extract_subworkload(w, sample)
+        sec = time_oracle(sub, sample, 1, 0)
+        stok = int(sub.path_q_len.astype(np.int64).sum())
+        out["cpu_baseline"] = {
+            "value": stok / sec, "unit": UNIT, "cores": oracle.host_cores(), "kind": "oracle",
+            "sample": f"{len(sample)} unique paths of {args.workload} ({int((sub.path_q_len > 1).sum())} verification, "
+                      f"{int((sub.path_q_len == 1).sum())} decode), {stok} query tokens, {sec:.1f} s"}
+
+    if rank == 0:
+        print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -277,13 +277,13 @@ extern "C" int32_t ss_dedup_paths(const int32_t* tok_ids, const int64_t* tok_off
   using namespace ss;
   using namespace ss::dedup;
   if (n_paths < 0 || !num_unique_out) return SS_ERR_INVALID_ARG;
-  if ((slot_in == nullptr) != (slot_out == nullptr)) return SS_ERR_INVALID_ARG;
   if (flags & ~SS_FLAG_WEAK_HASH) return SS_ERR_INVALID_ARG;
   cudaStream_t st = as_stream(stream);
   if (n_paths == 0) {
     SS_LAUNCH(zero_scalar_kernel, 1, 1, 0, st, num_unique_out);
     return SS_OK;
   }
+  if ((slot_in == nullptr) != (slot_out == nullptr)) return SS_ERR_INVALID_ARG;
   if (!tok_offsets || !canon_out || !path_to_unique_out || !unique_paths_out || !multiplicity_out || !workspace)
     return SS_ERR_INVALID_ARG;
   if (!tok_ids) return SS_ERR_INVALID_ARG;

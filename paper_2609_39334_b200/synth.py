@@ -336,9 +336,10 @@ def _decode(i, n, rng):
     return 1
 
 
-def make_config(idx: int, device="cpu", scale: float = 1.0, poison: bool = True) -> TreeWorkload:
-    """Config 1..5 of the benchmark list.  `scale` < 1 shrinks the number of problems (tests only)."""
-    seed = BASE_SEED + idx
+def make_config(idx: int, device="cpu", scale: float = 1.0, poison: bool = True, replica: int = 0) -> TreeWorkload:
+    """Config 1..5 of the benchmark list.  `scale` < 1 shrinks the number of problems (tests only); `replica`
+    selects a different seed for the same shapes (one replica per GPU in a multi-GPU run)."""
+    seed = BASE_SEED + idx + 1000 * replica
     if idx == 1:
         # 1 problem, 8 paths sharing a 256-token prefix, suffix U[0,64], decode; 12/2 heads; 2 of 8 identical
         return build_tree_workload("c1_tiny", seed, 12, 2, [256], [8], 1, (0, 64), _decode,
