@@ -97,6 +97,31 @@ int32_t ss_dedup_paths(const int32_t* tok_ids, const int64_t* tok_offsets, const
                        int32_t* slot_out, int32_t* num_unique_out, void* workspace, size_t workspace_bytes,
                        void* stream);
 
+/* ss_dedup_paths_static - ss_dedup_paths without a caller workspace and without any allocation.
+ *
+ * (The paper has no counterpart; this is a convenience of the library.)  It exists for callers that cannot ask
+ * the CUDA allocator for scratch when they need a deduplication pass - for instance a serving engine whose free
+ * HBM has all gone to its KV-cache pool, a scheduling loop that cannot afford the device-wide synchronisation an
+ * allocation may imply, or an embedded plug-in that is not permitted to allocate.  The scratch is a fixed 2 MiB
+ * array in device global memory that is part of the library image: every GPU that loads the library holds it
+ * until the process exits.
+ *
+ *   Arguments and results are those of ss_dedup_paths (same meaning, same layout, bit-identical outputs), minus
+ *   the workspace pair.  n_paths may be at most SS_DEDUP_STATIC_MAX_PATHS (65536); a larger value returns
+ *   SS_ERR_UNSUPPORTED and nothing is launched - use ss_dedup_paths with your own workspace then.
+ *   The call itself, and everything it calls, performs no cudaMalloc / cudaFree or other allocating routine.
+ *   The first call on each device looks up the array's device address (cudaGetSymbolAddress, with that device
+ *   current); make that first call outside any stream capture.
+ *   All calls on one device share the one array and the array keeps whatever the previous call left there (no
+ *   part of it needs clearing between calls).  Two calls whose kernels can overlap on the GPU - different
+ *   streams, or several host threads - race on it and give undefined results: serialise them.
+ * Errors: as ss_dedup_paths, plus SS_ERR_UNSUPPORTED for n_paths above the maximum. */
+#define SS_DEDUP_STATIC_MAX_PATHS 65536
+int32_t ss_dedup_paths_static(const int32_t* tok_ids, const int64_t* tok_offsets, const int64_t* ctx_key,
+                              const int32_t* slot_in, int32_t n_paths, uint32_t flags, int32_t* canon_out,
+                              int32_t* path_to_unique_out, int32_t* unique_paths_out, int32_t* multiplicity_out,
+                              int32_t* slot_out, int32_t* num_unique_out, void* stream);
+
 /* =========================================================================================================
  * ss_tree_attention - attention over a tree of candidate paths that share KV prefixes.
  *

@@ -28,11 +28,13 @@ SS_FLAG_FORCE_GENERIC = 0x2
 SS_FLAG_NO_TCGEN05 = 0x4
 SS_FLAG_WEAK_HASH = 0x8
 SS_MAX_DEPTH = 16
+SS_DEDUP_STATIC_MAX_PATHS = 65536
 
 EXPORTS = [
     "ss_status_string", "ss_last_device_status", "ss_dedup_workspace_bytes", "ss_dedup_paths",
     "ss_tree_attention_workspace_bytes", "ss_tree_attention", "ss_topk_workspace_bytes", "ss_topk_prune",
     "ss_launch_count", "ss_debug_umma_tile", "ss_profile_enable", "ss_profile_read",
+    "ss_dedup_paths_static",
 ]
 PHASES = ["plan", "tiles", "leaves", "generic", "merge"]
 
@@ -139,6 +141,19 @@ def ss_dedup_paths(tok_ids, tok_offsets, ctx_key, slot_in, n_paths, flags, canon
                               _stream(stream))
     if check:
         _check(rc, "ss_dedup_paths")
+    return rc
+
+
+def ss_dedup_paths_static(tok_ids, tok_offsets, ctx_key, slot_in, n_paths, flags, canon_out, path_to_unique_out,
+                          unique_paths_out, multiplicity_out, slot_out, num_unique_out, stream=None, check=True) -> int:
+    """ss_dedup_paths for callers that may not allocate: no workspace argument, the scratch is a fixed array inside
+    the library (at most SS_DEDUP_STATIC_MAX_PATHS paths; calls must not overlap on the GPU)."""
+    rc = lib().ss_dedup_paths_static(_ptr(tok_ids), _ptr(tok_offsets), _ptr(ctx_key), _ptr(slot_in),
+                                     ctypes.c_int32(n_paths), ctypes.c_uint32(flags), _ptr(canon_out),
+                                     _ptr(path_to_unique_out), _ptr(unique_paths_out), _ptr(multiplicity_out),
+                                     _ptr(slot_out), _ptr(num_unique_out), _stream(stream))
+    if check:
+        _check(rc, "ss_dedup_paths_static")
     return rc
 
 

@@ -322,3 +322,65 @@ extern "C" int32_t ss_dedup_paths(const int32_t* tok_ids, const int64_t* tok_off
             unique_paths_out, multiplicity_out, slot_out);
   return SS_OK;
 }
+
+// ---------------------------------------------------------------------------------------------------------
+// ss_dedup_paths_static: the same deduplication for callers that must not allocate device memory.
+//
+// Some hosts of this library cannot obtain scratch memory at the moment they need a deduplication pass: a serving
+// engine that has already handed all free HBM to its KV-cache pool (an allocation would fail, or shrink the cache),
+// a latency-critical scheduling loop in which the device-wide synchronisation hidden in an allocation is not
+// acceptable, or a plug-in that is simply not allowed to touch the allocator.  For them the scratch lives in the
+// library image itself: a fixed array in device global memory, present on every GPU that loads the library, from
+// load until the process ends.
+//
+// In host code the array's name below is only a handle for the runtime, not a device address; the address that
+// kernels can use is obtained once per device with cudaGetSymbolAddress (with that device current) and cached.
+// ---------------------------------------------------------------------------------------------------------
+namespace ss {
+namespace dedup {
+
+constexpr int kStaticMaxPaths = SS_DEDUP_STATIC_MAX_PATHS;
+constexpr size_t kStaticScratchBytes = 2u << 20;           // 2 MiB; layout(kStaticMaxPaths).total is about 1.8 MiB
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+static void* g_static_scratch_addr[kMaxDevices] = {nullptr};
+
+// Device address of the scratch array on the current device (looked up on the first call per device).
+static int32_t static_scratch_address(void** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); return SS_ERR_CUDA; }
+  if (dev < 0 || dev >= kMaxDevices) return SS_ERR_UNSUPPORTED;
+  if (!g_static_scratch_addr[dev]) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) {
+      (void)cudaGetLastError();
+      return SS_ERR_CUDA;
+    }
+    g_static_scratch_addr[dev] = ptr;
+  }
+  *out = g_static_scratch_addr[dev];
+  return SS_OK;
+}
+
+}  // namespace dedup
+}  // namespace ss
+
+extern "C" int32_t ss_dedup_paths_static(const int32_t* tok_ids, const int64_t* tok_offsets, const int64_t* ctx_key,
+                                         const int32_t* slot_in, int32_t n_paths, uint32_t flags, int32_t* canon_out,
+                                         int32_t* path_to_unique_out, int32_t* unique_paths_out,
+                                         int32_t* multiplicity_out, int32_t* slot_out, int32_t* num_unique_out,
+                                         void* stream) {
+  using namespace ss::dedup;
+  if (n_paths < 0) return SS_ERR_INVALID_ARG;
+  if (n_paths > kStaticMaxPaths) return SS_ERR_UNSUPPORTED;          // larger batches need ss_dedup_paths
+  if (layout(n_paths).total > kStaticScratchBytes) return SS_ERR_UNSUPPORTED;
+  void* scratch = nullptr;
+  const int32_t rc = static_scratch_address(&scratch);
+  if (rc != SS_OK) return rc;
+  // Nothing in the scratch has to start at zero: every region is fully written before it is read (histograms,
+  // keys, ranks), and the multiplicities that do start at zero are an output cleared by the rank kernel.
+  return ss_dedup_paths(tok_ids, tok_offsets, ctx_key, slot_in, n_paths, flags, canon_out, path_to_unique_out,
+                        unique_paths_out, multiplicity_out, slot_out, num_unique_out, scratch, kStaticScratchBytes,
+                        stream);
+}
