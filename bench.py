@@ -181,6 +181,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--profiler-range", action="store_true",
+                    help="bracket the timed region with cudaProfilerStart/Stop (for ncu --profile-from-start off)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
 
@@ -266,6 +268,8 @@ def main():
     B.ss_profile_enable(True)
     launches0 = B.ss_launch_count()
     sync_all()
+    if args.profiler_range:
+        torch.cuda.profiler.start()
     for i in range(args.steps):
         if flush is not None:
             flush.fill_(i & 0xff)       # evicts the pool from L2 between iterations (outside the timed events)
@@ -273,6 +277,8 @@ def main():
         pipe.step()
         ev[i][1].record()
     sync_all()
+    if args.profiler_range:
+        torch.cuda.profiler.stop()
     launches = B.ss_launch_count() - launches0
     B.ss_profile_enable(False)
     phase_ms, phase_calls = B.ss_profile_read()
@@ -309,7 +315,8 @@ def main():
         ach = work["tile_flops"] / (t_ms * 1e-3) / 1e12
         roofs["tiles"] = {"kernel": "tile_items_umma_kernel", "bound": "tensor", "achieved": ach, "peak": tensor_peak,
                           "unit": "TFLOP/s", "frac": ach / tensor_peak, "traffic": traffic.get("tiles"),
-                          "ms_per_launch": t_ms, "peak_kind": f"{peaks['source']} {'sustained' if long_step else 'burst'}"}
+                          "ms_per_launch": t_ms, "peak_kind": f"{peaks['source']} {'sustained' if long_step else 'burst'}",
+                          "ctas_per_sm": int(B.lib().ss_debug_tile_kernel_occupancy())}
     if phase_calls["leaves"]:
         t_ms = phase_ms["leaves"] / phase_calls["leaves"]
         ach = work["leaf_bytes"] / (t_ms * 1e-3) / 1e9

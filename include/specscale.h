@@ -247,6 +247,10 @@ int64_t ss_launch_count(void);
 int32_t ss_profile_enable(int32_t on);
 int32_t ss_profile_read(float* phase_ms /* host */, int64_t* phase_calls /* host */);
 
+/* CTAs of the tcgen05 tile kernel that fit one SM according to the CUDA occupancy query (0 before the first
+ * ss_tree_attention call that used the kernel).  Diagnostics; no paper counterpart. */
+int32_t ss_debug_tile_kernel_occupancy(void);
+
 /* One 128 x N x K bf16 tile product on the tcgen05 tensor cores, C[128][N] (fp32, row-major) = A[128][K] *
  * op(B), with the same shared-memory descriptors and TMEM read-out as the attention kernel.
  *   b_is_mn_major == 0: B is [N][K] row-major (the K-operand form, like keys);  C = A * B^T

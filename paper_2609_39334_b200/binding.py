@@ -34,7 +34,7 @@ EXPORTS = [
     "ss_status_string", "ss_last_device_status", "ss_dedup_workspace_bytes", "ss_dedup_paths",
     "ss_tree_attention_workspace_bytes", "ss_tree_attention", "ss_topk_workspace_bytes", "ss_topk_prune",
     "ss_launch_count", "ss_debug_umma_tile", "ss_profile_enable", "ss_profile_read",
-    "ss_dedup_paths_static",
+    "ss_dedup_paths_static", "ss_debug_tile_kernel_occupancy",
 ]
 PHASES = ["plan", "tiles", "leaves", "generic", "merge"]
 

@@ -28,6 +28,7 @@ constexpr int kUmmaThreads = 192;
 constexpr int kStages = 2;
 constexpr uint32_t kTmemCols = 256;
 constexpr uint32_t kColO = 128;
+constexpr float kLazyLog2 = 8.0f;              // the reference maximum moves only when exceeded by 2^8
 constexpr int kOffQ = 0;                       // [2 halves][128 rows][128 B]
 constexpr int kOffK = 32768;                   // kStages x [2 halves][64 rows][128 B]
 constexpr int kOffV = kOffK + kStages * 16384;
@@ -96,6 +97,7 @@ tile_items_umma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_
   const int n_items = P.hdr->n_tile_items;
   const int G = P.G;
   const float cl2 = P.scale_log2;
+  const float lazy_raw = kLazyLog2 / cl2;   // the lazy-rescale threshold in raw score units
 
   uint32_t g_tile = 0;      // tiles this CTA has processed (identical in every role)
   uint32_t q_uses = 0;      // items with at least one tile
@@ -164,9 +166,17 @@ tile_items_umma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_
             sr[c] = __float_as_uint(s);
             mx = fmaxf(mx, s);
           }
-          const float m_new = fmaxf(m, mx);
-          const float mc = m_new == -INFINITY ? 0.f : m_new * cl2;
-          const float alpha = ex2(m * cl2 - mc);                  // 0 when the row had no visible key so far
+          // Lazy reference maximum: exponentials are taken relative to m (not the running maximum); m only moves
+          // when the tile's maximum exceeds it by more than 2^kLazyLog2, so P stays <= 2^kLazyLog2 and the O
+          // accumulator in TMEM rarely needs rescaling.  out = O / l and lse = m*scale + ln l hold for any m.
+          const bool move = mx > m + lazy_raw;                    // also true for the first visible key (m = -inf)
+          float alpha = 1.f;
+          if (move) {
+            alpha = ex2((m - mx) * cl2);                          // 0 when the row had no visible key so far
+            m = mx;
+            l *= alpha;
+          }
+          const float mc = m == -INFINITY ? 0.f : m * cl2;
           float sum = 0.f;
           uint32_t pr[32];
 #pragma unroll
@@ -177,9 +187,7 @@ tile_items_umma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_
             __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
             pr[c >> 1] = *reinterpret_cast<uint32_t*>(&pk);
           }
-          l = l * alpha + sum;
-          const bool grew = (j > 0) && (m_new > m);
-          m = m_new;
+          l += sum;
 
           if (j > 0) {                                            // PV of the previous tile must be done before P / O change
             ok = mbar_wait(&C.pv_done, (gj - 1) & 1, abort_flag);
@@ -187,16 +195,20 @@ tile_items_umma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_
             if (!ok) break;
             tc_fence_after();
           }
-          if (__any_sync(0xffffffffu, grew)) {                    // rescale O (warp-collective TMEM access)
-            const float a = grew ? alpha : 1.f;
+          if (__any_sync(0xffffffffu, move && j > 0)) {           // rescale O (warp-collective TMEM access)
 #pragma unroll
-            for (int c0 = 0; c0 < kHeadDim; c0 += 32) {
-              uint32_t orow[32];
-              tmem_ld32(tmem + lane_base + kColO + c0, orow);
+            for (int c0 = 0; c0 < kHeadDim; c0 += 64) {
+              uint32_t o0[32], o1[32];
+              tmem_ld32(tmem + lane_base + kColO + c0, o0);
+              tmem_ld32(tmem + lane_base + kColO + c0 + 32, o1);
               tmem_wait_ld();
 #pragma unroll
-              for (int x = 0; x < 32; ++x) orow[x] = __float_as_uint(__uint_as_float(orow[x]) * a);
-              tmem_st32(tmem + lane_base + kColO + c0, orow);
+              for (int x = 0; x < 32; ++x) {
+                o0[x] = __float_as_uint(__uint_as_float(o0[x]) * alpha);
+                o1[x] = __float_as_uint(__uint_as_float(o1[x]) * alpha);
+              }
+              tmem_st32(tmem + lane_base + kColO + c0, o0);
+              tmem_st32(tmem + lane_base + kColO + c0 + 32, o1);
             }
             tmem_wait_st();
           }
@@ -304,6 +316,18 @@ tile_items_umma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_
         __syncwarp();
         const int n_seg = C.n_seg;
         bool ok = true;
+        // page of tile j handled by this lane -> row coordinate of its (page, kv head) block in the pool
+        auto page_coord = [&](int j) -> int {
+          const int pos0 = it.kv_begin + j * kKvTile;
+          const int n_pages = (min(kKvTile, it.kv_end - pos0) + kPage - 1) / kPage;
+          if (j >= n_tiles || lane >= n_pages) return 0;
+          const int vp = pos0 / kPage + lane;
+          int d = 0;
+          while (d + 1 < n_seg && vp >= C.seg_first_page[d + 1]) ++d;
+          const int64_t phys = P.node_pages[C.seg_page_off[d] + (vp - C.seg_first_page[d])];
+          return static_cast<int>((phys * P.page_stride + static_cast<int64_t>(it.g) * P.head_stride) >> 7);
+        };
+        int next_coord = page_coord(0);
         for (int j = 0; j < n_tiles && ok; ++j) {
           const uint32_t gj = g_tile + j;
           const int s = gj % kStages;
@@ -311,14 +335,8 @@ tile_items_umma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_
           const int pos0 = it.kv_begin + j * kKvTile;
           const int n_keys = min(kKvTile, it.kv_end - pos0);
           const int n_pages = (n_keys + kPage - 1) / kPage;
-          int coord_y = 0;
-          if (lane < n_pages) {
-            const int vp = pos0 / kPage + lane;
-            int d = 0;
-            while (d + 1 < n_seg && vp >= C.seg_first_page[d + 1]) ++d;
-            const int64_t phys = P.node_pages[C.seg_page_off[d] + (vp - C.seg_first_page[d])];
-            coord_y = static_cast<int>((phys * P.page_stride + static_cast<int64_t>(it.g) * P.head_stride) >> 7);
-          }
+          const int coord_y = next_coord;
+          next_coord = page_coord(j + 1);                         // in flight while this tile's slots are awaited
           // K
           if (u > 0) ok = mbar_wait(&C.k_empty[s], (u - 1) & 1, abort_flag);
           ok = __all_sync(0xffffffffu, ok);
@@ -405,6 +423,8 @@ tile_items_umma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_
   if (warp == 5) tmem_dealloc(tmem, kTmemCols);
 }
 
+int g_tile_kernel_occupancy = 0;   // CTAs per SM reported by the occupancy query (diagnostics)
+
 int32_t launch_tile_items_umma(const Params& P, cudaStream_t st, int sm_count) {
   static bool configured = false;
   static int ctas_per_sm = 1;
@@ -414,13 +434,18 @@ int32_t launch_tile_items_umma(const Params& P, cudaStream_t st, int sm_count) {
       (void)cudaGetLastError();
       return SS_ERR_CUDA;
     }
+    // two CTAs per SM need the largest shared-memory carve-out (2 x 113 KB + 2 KB reserved = 228 KB)
+    if (cudaFuncSetAttribute(tile_items_umma_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                             cudaSharedmemCarveoutMaxShared) != cudaSuccess)
+      (void)cudaGetLastError();
     int occ = 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, tile_items_umma_kernel, kUmmaThreads, kUmmaSmem) !=
             cudaSuccess || occ < 1) {
       (void)cudaGetLastError();
       occ = 1;
     }
-    ctas_per_sm = occ > 2 ? 2 : occ;             // TMEM: 2 x 256 columns per SM
+    g_tile_kernel_occupancy = occ;
+    ctas_per_sm = 2;                             // TMEM: 2 x 256 columns per SM; extra CTAs simply queue
     configured = true;
   }
   const int64_t rows = ((P.num_pages > 0 ? P.num_pages - 1 : 0) * P.page_stride + (P.Hkv - 1) * P.head_stride) / 128 + kPage;
@@ -435,3 +460,5 @@ int32_t launch_tile_items_umma(const Params& P, cudaStream_t st, int sm_count) {
 
 }  // namespace attn
 }  // namespace ss
+
+extern "C" int32_t ss_debug_tile_kernel_occupancy(void) { return ss::attn::g_tile_kernel_occupancy; }
