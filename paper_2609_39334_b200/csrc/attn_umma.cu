@@ -9,11 +9,14 @@
 //   warps 0-3  softmax + epilogue, one query row per thread = one TMEM lane
 //   warp 4     TMA producer: paged K / V boxes (one 16-token page x 64 dims each, 128-byte swizzle) into a
 //              2-stage ring, separate full/empty barriers for K and V
-//   warp 5     lane 0 issues the MMAs: S[b] = Q K^T (M128 N64 K16 x 8), O += P V (M128 N128 K16 x 4, V MN-major);
+//   warp 5     lane 0 issues the MMAs: S[b] = Q K^T (M128 N64 K16 x 8), O += P[b] V (M128 N128 K16 x 4, P in TMEM,
+//              V MN-major);
 //              the warp also owns the TMEM allocation (256 columns: two S buffers + O)
 // Per 64-key tile:  QK^T of tile j+1 is issued before PV of tile j, so the tensor pipe works on the next scores
-// while the softmax warps turn S[j] into P[j] (bf16, written to shared memory in the UMMA operand layout) and
-// rescale O in TMEM when a row maximum grew.  Softmax runs in the exp2 domain with the scale folded in.
+// while the softmax warps turn S[j] into P[j].  P (bf16) is written back into the TMEM columns of its own S buffer
+// and is the A operand of the PV product straight from TMEM, so it never touches shared memory.  The exponentials
+// use a lazily updated reference maximum, so the O accumulator in TMEM is rescaled only when a row maximum jumps
+// by more than 2^8.  Softmax runs in the exp2 domain with the scale folded in.
 // Every mbarrier wait is bounded; on expiry the CTA raises its abort flag, all roles fall through to the item-end
 // barrier, the CTA frees its TMEM and the kernel records SS_ERR_TIMEOUT.
 #include "attn_plan.cuh"
@@ -32,13 +35,15 @@ constexpr float kLazyLog2 = 8.0f;              // the reference maximum moves on
 constexpr int kOffQ = 0;                       // [2 halves][128 rows][128 B]
 constexpr int kOffK = 32768;                   // kStages x [2 halves][64 rows][128 B]
 constexpr int kOffV = kOffK + kStages * 16384;
-constexpr int kOffP = kOffV + kStages * 16384;  // [128 rows][128 B]
-constexpr int kOffCtrl = kOffP + 16384;
+constexpr int kOffCtrl = kOffV + kStages * 16384;
 constexpr int kUmmaSmem = kOffCtrl + 1024;
 
 struct Ctrl {
-  uint64_t q_full, k_full[kStages], v_full[kStages], k_empty[kStages], v_empty[kStages], s_full[2], s_empty[2], p_full,
-      pv_done;
+  // Parity waits are only safe when the waiter is never two completions away from the barrier's phase, hence:
+  // p_full is per S/P buffer (the softmax warps may run one tile ahead of the MMA thread), pv_done is waited only
+  // for the previous tile (it cannot lag further once S of the current tile exists), o_final fires once per item.
+  uint64_t q_full, k_full[kStages], v_full[kStages], k_empty[kStages], v_empty[kStages], s_full[2], p_full[2], pv_done,
+      o_final;
   uint32_t tmem_slot;
   int abort_flag;
   int item_idx;
@@ -82,9 +87,9 @@ tile_items_umma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_
       mbar_init(&C.k_full[s], 1); mbar_init(&C.v_full[s], 1);
       mbar_init(&C.k_empty[s], 1); mbar_init(&C.v_empty[s], 1);
     }
-    for (int b = 0; b < 2; ++b) { mbar_init(&C.s_full[b], 1); mbar_init(&C.s_empty[b], 128); }
-    mbar_init(&C.p_full, 128);
+    for (int b = 0; b < 2; ++b) { mbar_init(&C.s_full[b], 1); mbar_init(&C.p_full[b], 128); }
     mbar_init(&C.pv_done, 1);
+    mbar_init(&C.o_final, 1);
     fence_barrier_init();
     prefetch_tensormap(&tmap_k);
     prefetch_tensormap(&tmap_v);
@@ -154,18 +159,21 @@ tile_items_umma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_
           tmem_ld32(tmem + lane_base + b * 64, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
           tmem_ld32(tmem + lane_base + b * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
           tmem_wait_ld();
-          tc_fence_before();
-          mbar_arrive(&C.s_empty[b]);
 
           const int pos0 = it.kv_begin + j * kKvTile;
           const int nvis = limit_row - pos0;                      // visible columns of this tile for this row
-          float mx = -INFINITY;
+          if (!__all_sync(0xffffffffu, nvis >= kKvTile)) {        // causal tail or end of the source: mask
 #pragma unroll
-          for (int c = 0; c < 64; ++c) {
-            const float s = c < nvis ? __uint_as_float(sr[c]) : -INFINITY;
-            sr[c] = __float_as_uint(s);
-            mx = fmaxf(mx, s);
+            for (int c = 0; c < 64; ++c)
+              if (c >= nvis) sr[c] = 0xff800000u;                 // -inf
           }
+          float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+          for (int c = 0; c < 64; c += 4) {
+#pragma unroll
+            for (int x = 0; x < 4; ++x) mx4[x] = fmaxf(mx4[x], __uint_as_float(sr[c + x]));
+          }
+          const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
           // Lazy reference maximum: exponentials are taken relative to m (not the running maximum); m only moves
           // when the tile's maximum exceeds it by more than 2^kLazyLog2, so P stays <= 2^kLazyLog2 and the O
           // accumulator in TMEM rarely needs rescaling.  out = O / l and lse = m*scale + ln l hold for any m.
@@ -177,25 +185,23 @@ tile_items_umma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_
             l *= alpha;
           }
           const float mc = m == -INFINITY ? 0.f : m * cl2;
-          float sum = 0.f;
+          float sum4[4] = {0.f, 0.f, 0.f, 0.f};
           uint32_t pr[32];
 #pragma unroll
           for (int c = 0; c < 64; c += 2) {
             const float p0 = ex2(__uint_as_float(sr[c]) * cl2 - mc);
             const float p1 = ex2(__uint_as_float(sr[c + 1]) * cl2 - mc);
-            sum += p0 + p1;
+            sum4[(c >> 1) & 3] += p0 + p1;
             __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
             pr[c >> 1] = *reinterpret_cast<uint32_t*>(&pk);
           }
-          l += sum;
+          l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
 
-          if (j > 0) {                                            // PV of the previous tile must be done before P / O change
-            ok = mbar_wait(&C.pv_done, (gj - 1) & 1, abort_flag);
+          if (__any_sync(0xffffffffu, move && j > 0)) {           // rescale O (warp-collective TMEM access)
+            ok = mbar_wait(&C.pv_done, (gj - 1) & 1, abort_flag); // PV of the previous tile must have landed in O
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-          }
-          if (__any_sync(0xffffffffu, move && j > 0)) {           // rescale O (warp-collective TMEM access)
 #pragma unroll
             for (int c0 = 0; c0 < kHeadDim; c0 += 64) {
               uint32_t o0[32], o1[32];
@@ -226,17 +232,15 @@ tile_items_umma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_
               *reinterpret_cast<uint4*>(vs + (cc >> 3) * 8192 + r * 128 + (cc & 7) * 16) = make_uint4(0, 0, 0, 0);
             }
           }
-          // ---- P (bf16) into the A-operand layout ----------------------------------------------------------------
-#pragma unroll
-          for (int ch = 0; ch < 8; ++ch)
-            *reinterpret_cast<uint4*>(smem + kOffP + sw128_offset(row, ch)) =
-                make_uint4(pr[4 * ch], pr[4 * ch + 1], pr[4 * ch + 2], pr[4 * ch + 3]);
-          fence_proxy_async_smem();
+          // ---- P (bf16 pairs) over the first 32 columns of its own S buffer: the A operand of PV, read from TMEM ------
+          tmem_st32(tmem + lane_base + b * 64, pr);
+          tmem_wait_st();
+          if (n_keys < kKvTile) fence_proxy_async_smem();         // the V rows cleared above
           tc_fence_before();
-          mbar_arrive(&C.p_full);
+          mbar_arrive(&C.p_full[b]);
         }
         if (ok) {
-          ok = mbar_wait(&C.pv_done, (g_tile + n_tiles - 1) & 1, abort_flag);
+          ok = mbar_wait(&C.o_final, q_uses & 1, abort_flag);
           ok = __all_sync(0xffffffffu, ok);
           tc_fence_after();
         }
@@ -365,13 +369,13 @@ tile_items_umma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_
       // =================================================== MMA issuer ==========================================
       constexpr uint32_t idesc_qk = instr_desc_bf16(128, kKvTile, false);
       constexpr uint32_t idesc_pv = instr_desc_bf16(128, kHeadDim, true);
-      const uint32_t q_addr = smem_u32(smem + kOffQ), p_addr = smem_u32(smem + kOffP);
+      const uint32_t q_addr = smem_u32(smem + kOffQ);
       bool ok = mbar_wait(&C.q_full, q_uses & 1, abort_flag);
       auto issue_qk = [&](int j) -> bool {
         const uint32_t gj = g_tile + j;
         const int s = gj % kStages, b = gj & 1;
+        // S[b] / P[b] of tile gj-2 is free: PV(gj-2) was issued earlier by this thread and MMAs execute in order
         if (!mbar_wait(&C.k_full[s], (gj / kStages) & 1, abort_flag)) return false;
-        if (gj >= 2 && !mbar_wait(&C.s_empty[b], ((gj >> 1) - 1) & 1, abort_flag)) return false;
         tc_fence_after();
         const uint32_t k_addr = smem_u32(smem + kOffK + s * 16384);
 #pragma unroll
@@ -389,19 +393,20 @@ tile_items_umma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_
         if (j + 1 < n_tiles) ok = issue_qk(j + 1);
         if (!ok) break;
         const uint32_t gj = g_tile + j;
-        const int s = gj % kStages;
-        ok = mbar_wait(&C.v_full[s], (gj / kStages) & 1, abort_flag) && mbar_wait(&C.p_full, gj & 1, abort_flag);
+        const int s = gj % kStages, b = gj & 1;
+        ok = mbar_wait(&C.v_full[s], (gj / kStages) & 1, abort_flag) &&
+             mbar_wait(&C.p_full[b], (gj >> 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
         const uint32_t v_addr = smem_u32(smem + kOffV + s * 16384);
 #pragma unroll
         for (int kk = 0; kk < 4; ++kk) {
-          const uint64_t ad = smem_desc_sw128(p_addr + kk * 32, 0, 1024);
           const uint64_t bd = smem_desc_sw128(v_addr + kk * 2048, 8192, 1024);
-          mma_bf16_ss(tmem + kColO, ad, bd, idesc_pv, (j > 0 || kk > 0) ? 1u : 0u);
+          mma_bf16_ts(tmem + kColO, tmem + b * 64 + kk * 8, bd, idesc_pv, (j > 0 || kk > 0) ? 1u : 0u);
         }
         mma_commit(&C.v_empty[s]);
         mma_commit(&C.pv_done);
+        if (j + 1 == n_tiles) mma_commit(&C.o_final);
       }
     }
     // ---- item end: every role meets here, so the next item starts from a drained pipeline --------------------
