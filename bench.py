@@ -305,10 +305,13 @@ def main():
     long_step = total_ms > 1000.0
     tensor_peak = peaks["bf16_sustained"] if long_step else peaks["bf16_burst"]
     traffic = {}
-    tpath = os.path.join(ROOT, "profiles", "dram_traffic.json")
-    if os.path.exists(tpath):
+    tpath = os.path.join(ROOT, "profiles", "dram_traffic.txt")
+    if os.path.exists(tpath) and args.scale == 1.0:
         with open(tpath) as f:
-            traffic = json.load(f).get(args.workload, {})
+            for line in f:
+                parts = line.split()
+                if len(parts) == 3 and parts[0] == args.workload:
+                    traffic[parts[1]] = float(parts[2])
     roofs = {}
     if phase_calls["tiles"]:
         t_ms = phase_ms["tiles"] / phase_calls["tiles"]

@@ -380,3 +380,38 @@ def test_attention_device_errors_are_reported():
     pipe = DevicePipeline.__new__(DevicePipeline)
     with pytest.raises(B.SpecScaleError):
         DevicePipeline.__init__(pipe, deep, DEV)     # max_depth hint 18 > SS_MAX_DEPTH: rejected on the host
+
+
+# =========================================================================================================
+# full-size configuration 5 (the benchmark's workload, generated on the GPU): sampled outputs against the oracle
+# =========================================================================================================
+def test_config5_full_size_sampled_outputs():
+    w = synth.make_config(5, device=DEV)                    # 16384 paths, ~42 GB pool, both modes, 20 % duplicates
+    pipe = DevicePipeline(w, DEV)
+    pipe.step()
+    r = pipe.results()
+    ref = check_dedup(r, w)                                 # dedup / remap bit-exact on all 16384 paths
+    check_topk(r, w)
+    U = ref["num_unique"]
+    assert U < w.num_paths
+    uniq = ref["unique_paths"]
+    T = w.path_q_len[uniq]
+    lens = w.node_kv_len[w.path_leaf_node[uniq]]
+    rng = np.random.default_rng(5)
+    ver, dec = np.nonzero(T > 1)[0], np.nonzero(T == 1)[0]
+    pick = set(int(x) for x in rng.choice(ver, 14, replace=False)) | set(int(x) for x in rng.choice(dec, 40, replace=False))
+    pick |= {int(dec[lens[dec].argmin()]), int(dec[lens[dec].argmax()]), int(ver[lens[ver].argmin()]),
+             int(ver[lens[ver].argmax()]), 0, U - 1}
+    dup_u = np.nonzero(ref["multiplicity"] > 1)[0]
+    pick |= {int(dup_u[0]), int(dup_u[-1])}
+    sel = np.asarray(sorted(pick))
+    sub = synth.extract_subworkload(w, uniq[sel])           # the needed pages and query rows, copied to the host
+    o_ref, l_ref = oracle.tree_attention_workload(sub)
+    off = np.concatenate([[0], np.cumsum(T.astype(np.int64))])
+    rows = np.concatenate([np.arange(off[i], off[i + 1]) for i in sel])
+    out, lse = r["out"][rows], r["lse"][rows]
+    assert np.isfinite(out).all()
+    err = np.abs(out - o_ref)
+    lerr = np.abs(lse - l_ref).max()
+    assert err.max() <= OUT_MAX and err.mean() <= OUT_MEAN and lerr <= LSE_MAX, (err.max(), err.mean(), lerr)
+    assert err.max() <= TIGHT_OUT_MAX and err.mean() <= TIGHT_OUT_MEAN and lerr <= TIGHT_LSE, (err.max(), err.mean(), lerr)
