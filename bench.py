@@ -237,7 +237,8 @@ def main():
     B.lib()
 
     # every rank its own problems: same shapes, different seed
-    w = synth.make_config(cfg_idx, device=dev, scale=args.scale, poison=True, replica=rank)
+    from paper_2609_39334_b200 import replicas
+    w = replicas.replica_workload(synth.make_config, cfg_idx, rank, device=dev, scale=args.scale, poison=True)
     pipe = DevicePipeline(w, dev)
     kv_bytes = pipe.kv_pool.numel() * 2
     flush = None
@@ -284,11 +285,7 @@ def main():
     phase_ms, phase_calls = B.ss_profile_read()
     clk = clocks.stop() if rank == 0 else None
     step_ms = [a.elapsed_time(b) for a, b in ev]
-    total_ms = float(sum(step_ms))
-    if dist is not None:
-        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = replicas.max_over_ranks(float(sum(step_ms)), dev)
     ms_per_step = total_ms / args.steps
     st = B.ss_last_device_status(pipe.attn_ws)
     if st != B.SS_OK:
@@ -298,7 +295,7 @@ def main():
     unique_paths = pipe.unique_paths[:U].cpu().numpy()
     work = algorithmic_work(w, unique_paths)
     tokens = work["tokens"]
-    value = world * tokens / (ms_per_step * 1e-3)
+    value = replicas.whole_job_rate(tokens, ms_per_step)
 
     # ---- roofline of the attention kernels (per launch, CUDA events on the launching stream) -----------------
     peaks = load_peaks()
@@ -374,11 +371,7 @@ def main():
             e2e_step()
         e1.record()
         sync_all()
-        e2e_ms = e0.elapsed_time(e1) / n_e2e
-        if dist is not None:
-            t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
+        e2e_ms = replicas.max_over_ranks(e0.elapsed_time(e1) / n_e2e, dev)
         out["e2e"] = {"value": world * tokens / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
                       "d2h_bytes_per_step": int(d2h), "ms_per_step": e2e_ms, "steps": n_e2e,
                       "note": "KV pool stays resident (it is the cache); candidates, queries and scores come from "
