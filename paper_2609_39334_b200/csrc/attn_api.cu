@@ -99,8 +99,8 @@ static Layout carve(const ss_attn_desc_t* d, char* base, Params* P) {
   char* hdr = take(sizeof(PlanHeader));
   char* node_arrays[11];
   for (int i = 0; i < 11; ++i) node_arrays[i] = take(N * 4);
-  char* path_arrays[4];
-  for (int i = 0; i < 4; ++i) path_arrays[i] = take(NP * 4);
+  char* path_arrays[6];
+  for (int i = 0; i < 6; ++i) path_arrays[i] = take(NP * 4);
   char* dec_tok = take((static_cast<size_t>(cap_dec) + 1) * 4);
   char* dec_slot = take((static_cast<size_t>(cap_dec) + 1) * 4);
   char* tiles = take(static_cast<size_t>(caps.tile_items) * sizeof(TileItem));
@@ -112,8 +112,9 @@ static Layout carve(const ss_attn_desc_t* d, char* base, Params* P) {
     int32_t** np[11] = {&P->node_start, &P->node_depth, &P->node_first, &P->node_last, &P->node_npaths, &P->node_ndec,
                         &P->node_own_slots, &P->node_level_off, &P->node_item_base, &P->node_splits, &P->node_split_len};
     for (int i = 0; i < 11; ++i) *np[i] = reinterpret_cast<int32_t*>(node_arrays[i]);
-    int32_t** pp[4] = {&P->path_class, &P->path_kv_len, &P->path_dec_rank, &P->path_scan};
-    for (int i = 0; i < 4; ++i) *pp[i] = reinterpret_cast<int32_t*>(path_arrays[i]);
+    int32_t** pp[6] = {&P->path_class, &P->path_kv_len, &P->path_dec_rank, &P->path_slot_base, &P->path_leaf_base,
+                       &P->path_chain_base};
+    for (int i = 0; i < 6; ++i) *pp[i] = reinterpret_cast<int32_t*>(path_arrays[i]);
     P->dec_tok = reinterpret_cast<int32_t*>(dec_tok);
     P->dec_slot_base = reinterpret_cast<int32_t*>(dec_slot);
     P->tile_items = reinterpret_cast<TileItem*>(tiles);

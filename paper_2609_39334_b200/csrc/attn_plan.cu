@@ -1,49 +1,58 @@
-// Device-side planner of ss_tree_attention: one block turns the tree + per-path arrays into work lists
-// (tile items, leaf items), partial-slot assignments and per-path classes.  Running it on the device means
-// the live path count can come straight from ss_dedup_paths without a host round trip.
+// Device-side planner of ss_tree_attention: turns the tree + per-path arrays into work lists (tile items, leaf
+// items), partial-slot assignments and per-path classes.  Running it on the device means the live path count can
+// come straight from ss_dedup_paths without a host round trip.  Four small launches on the caller's stream:
+//   plan_nodes   (grid over nodes)   depth and prefix length of every node, range checks, counters reset
+//   plan_paths   (grid over paths)   class and key length of every path, membership counts of its chain nodes
+//   plan_scan    (one block)         every prefix sum: decode ranks, per-node tile items and KV splits, partial
+//                                    slots, leaf items, chain items; capacity checks; totals into the header
+//   plan_emit    (grid)              writes the item lists and the per-decode-token arrays
+// The header (status word first) is cleared by the host-side launcher before plan_nodes.
 #include "attn_plan.cuh"
 
 namespace ss {
 namespace attn {
 
-constexpr int kPlanThreads = 1024;
+constexpr int kScanThreads = 1024;
+constexpr int kGridThreads = 256;
 
-// In-place exclusive scan of a[0..n) by the whole block; returns the total to every thread.
+// In-place exclusive scan of a[0..n) by one whole block: every thread sums a contiguous chunk, the chunk sums are
+// scanned across the block, then every thread rewrites its chunk.  Returns the total to every thread.
 __device__ int block_excl_scan(int32_t* a, int n) {
   __shared__ int warp_tot[32];
-  __shared__ int carry_s;
+  __shared__ int total_s;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  const int chunk = (n + blockDim.x - 1) / blockDim.x;
+  const int lo = min(n, static_cast<int>(threadIdx.x) * chunk), hi = min(n, lo + chunk);
   __syncthreads();
-  if (threadIdx.x == 0) carry_s = 0;
+  int sum = 0;
+  for (int i = lo; i < hi; ++i) sum += a[i];
+  int x = sum;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int y = __shfl_up_sync(0xffffffffu, x, o);
+    if (lane >= o) x += y;
+  }
+  if (lane == 31) warp_tot[warp] = x;
   __syncthreads();
-  for (int base = 0; base < n; base += blockDim.x) {
-    const int i = base + threadIdx.x;
-    const int v = i < n ? a[i] : 0;
-    int x = v;
+  if (warp == 0) {
+    int t = lane < nw ? warp_tot[lane] : 0;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-      const int y = __shfl_up_sync(0xffffffffu, x, o);
-      if (lane >= o) x += y;
+      const int y = __shfl_up_sync(0xffffffffu, t, o);
+      if (lane >= o) t += y;
     }
-    if (lane == 31) warp_tot[warp] = x;
-    __syncthreads();
-    if (warp == 0) {
-      int t = lane < nw ? warp_tot[lane] : 0;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int y = __shfl_up_sync(0xffffffffu, t, o);
-        if (lane >= o) t += y;
-      }
-      warp_tot[lane] = t;
-    }
-    __syncthreads();
-    const int before = carry_s + (warp ? warp_tot[warp - 1] : 0) + x - v;
-    if (i < n) a[i] = before;
-    __syncthreads();
-    if (threadIdx.x == blockDim.x - 1) carry_s = before + v;
-    __syncthreads();
+    warp_tot[lane] = t;
+    if (lane == 31) total_s = t;
   }
-  return carry_s;
+  __syncthreads();
+  int run = (warp ? warp_tot[warp - 1] : 0) + x - sum;
+  for (int i = lo; i < hi; ++i) {
+    const int v = a[i];
+    a[i] = run;
+    run += v;
+  }
+  __syncthreads();
+  return total_s;
 }
 
 // Block-uniform read of the status word (every thread gets the same answer, so an early return cannot leave
@@ -51,42 +60,29 @@ __device__ int block_excl_scan(int32_t* a, int n) {
 __device__ bool block_failed(const PlanHeader* hdr) {
   __shared__ int s_status;
   __syncthreads();
-  if (threadIdx.x == 0) s_status = hdr->status;
+  if (threadIdx.x == 0) s_status = *reinterpret_cast<const volatile int32_t*>(&hdr->status);
   __syncthreads();
   return s_status != SS_OK;
 }
 
-__global__ void __launch_bounds__(kPlanThreads) plan_kernel(const Params P) {
-  __shared__ int s_live, s_total_tiles, s_generic;
-  PlanHeader* hdr = P.hdr;
-  const int tid = threadIdx.x, nt = blockDim.x;
-  if (tid == 0) {
-    int live = P.num_paths;
-    if (P.num_paths_dev) {
-      live = *P.num_paths_dev;
-      if (live < 0) live = 0;
-      if (live > P.num_paths) live = P.num_paths;
-    }
-    s_live = live;
-    s_total_tiles = 0;
-    s_generic = 0;
-    hdr->status = SS_OK;
-    hdr->live_paths = live;
-    hdr->n_dec = 0;
-    hdr->n_tile_items = 0;
-    hdr->n_leaf_items = 0;
-    hdr->n_slots = 0;
-    hdr->n_generic_rows = 0;
-    hdr->tile_counter = 0;
-    hdr->leaf_counter = 0;
+__device__ __forceinline__ int live_paths(const Params& P) {
+  int live = P.num_paths;
+  if (P.num_paths_dev) {
+    live = *P.num_paths_dev;
+    if (live < 0) live = 0;
+    if (live > P.num_paths) live = P.num_paths;
   }
-  __syncthreads();
-  const int live = s_live;
-  const int N = P.num_nodes;
-  const bool force_generic = (P.flags & SS_FLAG_FORCE_GENERIC) != 0;
+  return live;
+}
 
-  // ---- nodes: depth and number of keys before the node ---------------------------------------------------
-  for (int n = tid; n < N; n += nt) {
+// ---- nodes: depth and number of keys before the node -------------------------------------------------------------
+__global__ void __launch_bounds__(kGridThreads) plan_nodes_kernel(const Params P) {
+  PlanHeader* hdr = P.hdr;
+  const int64_t gtid = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  const int64_t gsize = static_cast<int64_t>(gridDim.x) * blockDim.x;
+  if (gtid == 0) hdr->live_paths = live_paths(P);
+  for (int64_t n64 = gtid; n64 < P.num_nodes; n64 += gsize) {
+    const int n = static_cast<int>(n64);
     int d = 0, start = 0;
     int a = P.node_parent[n];
     bool bad = (a >= n || a < -1 || P.node_kv_len[n] < 0);
@@ -111,22 +107,29 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(const Params P) {
     P.node_ndec[n] = 0;
   }
   if (P.flags & SS_FLAG_VALIDATE) {
-    for (int64_t i = tid; i < P.total_node_pages; i += nt) {
+    for (int64_t i = gtid; i < P.total_node_pages; i += gsize) {
       const int pg = P.node_pages[i];
       if (pg < 0 || pg >= P.num_pages) set_status(&hdr->status, SS_ERR_BAD_INPUT);
     }
   }
-  if (block_failed(hdr)) return;
+}
 
-  // ---- paths: class, kv length, membership counts of every chain node ---------------------------------------
-  for (int p = tid; p < live; p += nt) {
+// ---- paths: class, kv length, membership counts of every chain node ------------------------------------------------
+__global__ void __launch_bounds__(kGridThreads) plan_paths_kernel(const Params P) {
+  PlanHeader* hdr = P.hdr;
+  if (hdr->status != SS_OK) return;          // no barrier in this kernel: a per-thread return is safe
+  const int live = hdr->live_paths;
+  const int N = P.num_nodes;
+  const bool force_generic = (P.flags & SS_FLAG_FORCE_GENERIC) != 0;
+  const int64_t gsize = static_cast<int64_t>(gridDim.x) * blockDim.x;
+  for (int64_t p64 = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; p64 < live; p64 += gsize) {
+    const int p = static_cast<int>(p64);
     const int leaf = P.path_leaf_node[p];
     const int T = P.path_q_len[p];
     if (leaf < 0 || leaf >= N || T < 1 || P.q_offsets[p + 1] - P.q_offsets[p] != T || P.q_offsets[p] < 0 ||
         P.q_offsets[p + 1] > P.total_q) {
       set_status(&hdr->status, SS_ERR_BAD_INPUT);
       P.path_class[p] = kClassGeneric;
-      P.path_scan[p] = 0;
       continue;
     }
     bool inner_whole_pages = true;
@@ -138,8 +141,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(const Params P) {
     else cls = inner_whole_pages ? kClassChain : kClassGeneric;
     P.path_class[p] = cls;
     P.path_kv_len[p] = P.node_start[leaf] + P.node_kv_len[leaf];
-    P.path_scan[p] = (cls == kClassDecode) ? 1 : 0;
-    if (cls == kClassGeneric) atomicAdd(&s_generic, T);
+    if (cls == kClassGeneric) atomicAdd(&hdr->n_generic_rows, T);
     for (int a = leaf; a >= 0; a = P.node_parent[a]) {
       atomicMin(&P.node_first[a], p);
       atomicMax(&P.node_last[a], p);
@@ -147,23 +149,29 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(const Params P) {
       if (cls == kClassDecode) atomicAdd(&P.node_ndec[a], 1);
     }
   }
-  if (block_failed(hdr)) return;
+}
 
-  // ---- decode ranks ---------------------------------------------------------------------------------------------
-  for (int p = tid; p < live; p += nt) P.path_dec_rank[p] = P.path_scan[p];
+// ---- every prefix sum -------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kScanThreads) plan_scan_kernel(const Params P) {
+  __shared__ int s_total_tiles;
+  PlanHeader* hdr = P.hdr;
+  if (block_failed(hdr)) return;
+  const int tid = threadIdx.x, nt = blockDim.x;
+  const int live = hdr->live_paths;
+  const int N = P.num_nodes;
+  const int tpt = P.tok_per_tile;
+  if (tid == 0) s_total_tiles = 0;
+
+  // decode ranks
+  for (int p = tid; p < live; p += nt) P.path_dec_rank[p] = (P.path_class[p] == kClassDecode) ? 1 : 0;
   const int n_dec = block_excl_scan(P.path_dec_rank, live);
   if (tid == 0) {
     P.path_dec_rank[live] = n_dec;
     hdr->n_dec = n_dec;
-    hdr->n_generic_rows = s_generic;
     if (n_dec > P.caps.dec) set_status(&hdr->status, SS_ERR_WORKSPACE_TOO_SMALL);
   }
-  if (block_failed(hdr)) return;
-  for (int p = tid; p < live; p += nt)
-    if (P.path_class[p] == kClassDecode) P.dec_tok[P.path_dec_rank[p]] = static_cast<int32_t>(P.q_offsets[p]);
 
-  // ---- nodes: role, tiles ---------------------------------------------------------------------------------------
-  const int tpt = P.tok_per_tile;
+  // nodes: role, tiles
   for (int n = tid; n < N; n += nt) {
     const int np = P.node_npaths[n];
     if (np > 0 && P.node_last[n] - P.node_first[n] + 1 != np) set_status(&hdr->status, SS_ERR_BAD_INPUT);
@@ -179,7 +187,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(const Params P) {
   if (block_failed(hdr)) return;
   const int total_tiles = s_total_tiles * P.Hkv;
   for (int n = tid; n < N; n += nt) {
-    const int np = P.node_npaths[n], nd = P.node_ndec[n], len = P.node_kv_len[n];
+    const int nd = P.node_ndec[n], len = P.node_kv_len[n];
     const int tiles = P.node_item_base[n];
     int splits = 1, own = 0, split_len = len;
     if (nd > 0 && len > 0) {
@@ -199,7 +207,6 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(const Params P) {
         own = splits;
       }
     }
-    (void)np;
     P.node_splits[n] = splits;
     P.node_split_len[n] = split_len;
     P.node_own_slots[n] = own;
@@ -214,76 +221,98 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(const Params P) {
   const int n_stacked = block_excl_scan(P.node_item_base, N);
   if (tid == 0) P.node_item_base[N] = n_stacked;
 
-  // ---- decode paths: partial slots and leaf items ---------------------------------------------------------------
+  // decode paths: partial slots, leaf items; chain paths: tile items
   for (int p = tid; p < live; p += nt) {
-    int s = 0;
-    if (P.path_class[p] == kClassDecode) {
+    int slots = 0, leaf_items = 0, chain_items = 0;
+    const int cls = P.path_class[p];
+    if (cls == kClassDecode) {
       const int leaf = P.path_leaf_node[p];
-      s = P.node_level_off[leaf] + P.node_own_slots[leaf];
+      slots = P.node_level_off[leaf] + P.node_own_slots[leaf];
+      if (P.node_npaths[leaf] == 1 && P.node_kv_len[leaf] > 0)
+        leaf_items = ceil_div(P.node_kv_len[leaf], kLeafChunk) * P.Hkv;
+    } else if (cls == kClassChain) {
+      chain_items = ceil_div(P.path_q_len[p], tpt) * P.Hkv;
     }
-    P.path_scan[p] = s;
+    P.path_slot_base[p] = slots;
+    P.path_leaf_base[p] = leaf_items;
+    P.path_chain_base[p] = chain_items;
   }
-  const int n_slots = block_excl_scan(P.path_scan, live);
-  for (int p = tid; p < live; p += nt)
-    if (P.path_class[p] == kClassDecode) P.dec_slot_base[P.path_dec_rank[p]] = P.path_scan[p];
+  const int n_slots = block_excl_scan(P.path_slot_base, live);
+  const int n_leaf_items = block_excl_scan(P.path_leaf_base, live);
+  const int n_chain = block_excl_scan(P.path_chain_base, live);
   if (tid == 0) {
-    P.dec_slot_base[n_dec] = n_slots;
     hdr->n_slots = n_slots;
-    if (n_slots > P.caps.slots) set_status(&hdr->status, SS_ERR_WORKSPACE_TOO_SMALL);
-  }
-  __syncthreads();
-  // leaf items
-  for (int p = tid; p < live; p += nt) {
-    int c = 0;
-    if (P.path_class[p] == kClassDecode) {
-      const int leaf = P.path_leaf_node[p];
-      const bool leaf_only = (P.node_npaths[leaf] == 1);
-      if (leaf_only && P.node_kv_len[leaf] > 0) c = ceil_div(P.node_kv_len[leaf], kLeafChunk) * P.Hkv;
+    hdr->n_stacked_items = n_stacked;
+    if (n_slots > P.caps.slots || n_leaf_items > P.caps.leaf_items || n_stacked + n_chain > P.caps.tile_items) {
+      set_status(&hdr->status, SS_ERR_WORKSPACE_TOO_SMALL);     // the executors see the status and do nothing
+    } else {
+      hdr->n_leaf_items = n_leaf_items;
+      hdr->n_tile_items = n_stacked + n_chain;
     }
-    P.path_scan[p] = c;
   }
-  const int n_leaf_items = block_excl_scan(P.path_scan, live);
-  if (tid == 0) {
-    hdr->n_leaf_items = n_leaf_items;
-    if (n_leaf_items > P.caps.leaf_items) set_status(&hdr->status, SS_ERR_WORKSPACE_TOO_SMALL);
-  }
-  if (block_failed(hdr)) return;
-  for (int p = tid; p < live; p += nt) {
-    if (P.path_class[p] != kClassDecode) continue;
-    const int leaf = P.path_leaf_node[p];
-    const int len = P.node_kv_len[leaf];
-    if (!(P.node_npaths[leaf] == 1 && len > 0)) continue;
-    const int chunks = ceil_div(len, kLeafChunk);
-    int e = P.path_scan[p];
-    const int slot0 = P.dec_slot_base[P.path_dec_rank[p]] + P.node_level_off[leaf];
-    for (int c = 0; c < chunks; ++c)
-      for (int g = 0; g < P.Hkv; ++g) {
-        LeafItem it;
-        it.q_row = static_cast<int32_t>(P.q_offsets[p]);
-        it.node = leaf;
-        it.g = g;
-        it.kv_begin = c * kLeafChunk;
-        it.kv_end = min(len, (c + 1) * kLeafChunk);
-        it.slot = slot0 + c;
-        it.pad0 = it.pad1 = 0;
-        P.leaf_items[e++] = it;
-      }
-  }
-  __syncthreads();
+}
 
-  // ---- chain paths: tile items ----------------------------------------------------------------------------------
-  for (int p = tid; p < live; p += nt)
-    P.path_scan[p] = (P.path_class[p] == kClassChain) ? ceil_div(P.path_q_len[p], tpt) * P.Hkv : 0;
-  const int n_chain = block_excl_scan(P.path_scan, live);
-  const int n_items = n_stacked + n_chain;
-  if (tid == 0) {
-    hdr->n_tile_items = n_items;
-    if (n_items > P.caps.tile_items) set_status(&hdr->status, SS_ERR_WORKSPACE_TOO_SMALL);
+// ---- item lists ---------------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kGridThreads) plan_emit_kernel(const Params P) {
+  PlanHeader* hdr = P.hdr;
+  if (hdr->status != SS_OK) return;          // no barrier in this kernel
+  const int live = hdr->live_paths;
+  const int N = P.num_nodes;
+  const int tpt = P.tok_per_tile;
+  const int n_stacked = hdr->n_stacked_items;
+  const int64_t gtid = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  const int64_t gsize = static_cast<int64_t>(gridDim.x) * blockDim.x;
+  if (gtid == 0) P.dec_slot_base[hdr->n_dec] = hdr->n_slots;
+
+  for (int64_t p64 = gtid; p64 < live; p64 += gsize) {
+    const int p = static_cast<int>(p64);
+    const int cls = P.path_class[p];
+    if (cls == kClassDecode) {
+      const int rank = P.path_dec_rank[p];
+      const int leaf = P.path_leaf_node[p];
+      const int len = P.node_kv_len[leaf];
+      P.dec_tok[rank] = static_cast<int32_t>(P.q_offsets[p]);
+      P.dec_slot_base[rank] = P.path_slot_base[p];
+      if (!(P.node_npaths[leaf] == 1 && len > 0)) continue;
+      const int chunks = ceil_div(len, kLeafChunk);
+      int e = P.path_leaf_base[p];
+      const int slot0 = P.path_slot_base[p] + P.node_level_off[leaf];
+      for (int c = 0; c < chunks; ++c)
+        for (int g = 0; g < P.Hkv; ++g) {
+          LeafItem it;
+          it.q_row = static_cast<int32_t>(P.q_offsets[p]);
+          it.node = leaf;
+          it.g = g;
+          it.kv_begin = c * kLeafChunk;
+          it.kv_end = min(len, (c + 1) * kLeafChunk);
+          it.slot = slot0 + c;
+          it.pad0 = it.pad1 = 0;
+          P.leaf_items[e++] = it;
+        }
+    } else if (cls == kClassChain) {
+      const int T = P.path_q_len[p];
+      const int L = P.path_kv_len[p];
+      const int tiles = ceil_div(T, tpt);
+      int e = n_stacked + P.path_chain_base[p];
+      for (int g = 0; g < P.Hkv; ++g)
+        for (int t = 0; t < tiles; ++t) {
+          TileItem it;
+          it.node = P.path_leaf_node[p];
+          it.tok0 = static_cast<int32_t>(P.q_offsets[p]) + t * tpt;
+          it.n_tok = min(tpt, T - t * tpt);
+          it.kind_g = (kItemChain << 16) | g;
+          it.kv_begin = 0;
+          it.limit0 = L - T + t * tpt + 1;
+          it.kv_end = max(0, min(L, it.limit0 + it.n_tok - 1));
+          it.slot_off = -1;
+          P.tile_items[e++] = it;
+        }
+    }
   }
-  if (block_failed(hdr)) return;
 
   // stacked items: item e -> node by binary search over the exclusive scan of per-node item counts
-  for (int e = tid; e < n_stacked; e += nt) {
+  for (int64_t e64 = gtid; e64 < n_stacked; e64 += gsize) {
+    const int e = static_cast<int>(e64);
     int lo = 0, hi = N;                       // last n with base[n] <= e and base[n+1] > e
     while (hi - lo > 1) {
       const int mid = (lo + hi) >> 1;
@@ -310,30 +339,21 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(const Params P) {
     it.slot_off = P.node_level_off[n] + split;
     P.tile_items[e] = it;
   }
-  for (int p = tid; p < live; p += nt) {
-    if (P.path_class[p] != kClassChain) continue;
-    const int T = P.path_q_len[p];
-    const int L = P.path_kv_len[p];
-    const int tiles = ceil_div(T, tpt);
-    int e = n_stacked + P.path_scan[p];
-    for (int g = 0; g < P.Hkv; ++g)
-      for (int t = 0; t < tiles; ++t) {
-        TileItem it;
-        it.node = P.path_leaf_node[p];
-        it.tok0 = static_cast<int32_t>(P.q_offsets[p]) + t * tpt;
-        it.n_tok = min(tpt, T - t * tpt);
-        it.kind_g = (kItemChain << 16) | g;
-        it.kv_begin = 0;
-        it.limit0 = L - T + t * tpt + 1;
-        it.kv_end = max(0, min(L, it.limit0 + it.n_tok - 1));
-        it.slot_off = -1;
-        P.tile_items[e++] = it;
-      }
-  }
 }
 
 int32_t launch_plan(const Params& P, cudaStream_t st) {
-  SS_LAUNCH(plan_kernel, 1, kPlanThreads, 0, st, P);
+  if (cudaMemsetAsync(P.hdr, 0, sizeof(PlanHeader), st) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return SS_ERR_CUDA;
+  }
+  const int64_t work = P.num_nodes > P.num_paths ? P.num_nodes : P.num_paths;
+  int blocks = static_cast<int>((work + kGridThreads - 1) / kGridThreads);
+  if (blocks < 1) blocks = 1;
+  if (blocks > 1184) blocks = 1184;
+  SS_LAUNCH(plan_nodes_kernel, blocks, kGridThreads, 0, st, P);
+  SS_LAUNCH(plan_paths_kernel, blocks, kGridThreads, 0, st, P);
+  SS_LAUNCH(plan_scan_kernel, 1, kScanThreads, 0, st, P);
+  SS_LAUNCH(plan_emit_kernel, blocks, kGridThreads, 0, st, P);
   return SS_OK;
 }
 

@@ -60,7 +60,8 @@ struct PlanHeader {       // first bytes of the workspace; status MUST be the fi
   int32_t n_generic_rows; // > 0 if any path is GENERIC
   int32_t tile_counter;   // work-stealing counters (reset by the planner)
   int32_t leaf_counter;
-  int32_t pad[7];
+  int32_t n_stacked_items; // tile items [0, n_stacked_items) are stacked items, the rest chain items
+  int32_t pad[6];
 };
 
 struct Caps {             // host-computed capacities of the plan arrays
@@ -93,7 +94,7 @@ struct Params {
   PlanHeader* hdr;
   int32_t *node_start, *node_depth, *node_first, *node_last, *node_npaths, *node_ndec, *node_own_slots,
       *node_level_off, *node_item_base, *node_splits, *node_split_len;
-  int32_t *path_class, *path_kv_len, *path_dec_rank, *path_scan;
+  int32_t *path_class, *path_kv_len, *path_dec_rank, *path_slot_base, *path_leaf_base, *path_chain_base;
   int32_t *dec_tok, *dec_slot_base;
   TileItem* tile_items;
   LeafItem* leaf_items;
