@@ -38,6 +38,7 @@ def _load():
             lib.ss_oracle_dedup.restype = ctypes.c_int32
             lib.ss_oracle_tree_attention.restype = ctypes.c_int32
             lib.ss_oracle_topk.restype = None
+            lib.ss_oracle_early_prune.restype = None
             _lib = lib
     return _lib
 
@@ -159,3 +160,21 @@ def topk(scores, seg_offsets, k):
     sc = scores if n else np.zeros(1, np.float32)
     lib.ss_oracle_topk(_p(sc), _p(seg_offsets), ctypes.c_int32(n_seg), ctypes.c_int32(k), _p(surv), _p(keep))
     return surv[:n_seg, :k].reshape(n_seg, k), keep[:n]
+
+
+def early_prune(scores, verified, seg_offsets, k):
+    """-> (pruned uint8 [N], selected int32 [P][k] (-1 padded), final uint8 [P])."""
+    lib = _load()
+    scores = _c(scores, np.float32)
+    verified = _c(verified, np.uint8)
+    seg_offsets = _c(seg_offsets, np.int32)
+    n_seg = int(seg_offsets.shape[0]) - 1
+    n = int(scores.shape[0])
+    pruned = np.zeros(max(n, 1), np.uint8)
+    sel = np.full((max(n_seg, 1), max(k, 1)), -1, np.int32)
+    fin = np.zeros(max(n_seg, 1), np.uint8)
+    sc = scores if n else np.zeros(1, np.float32)
+    ve = verified if n else np.zeros(1, np.uint8)
+    lib.ss_oracle_early_prune(_p(sc), _p(ve), _p(seg_offsets), ctypes.c_int32(n_seg), ctypes.c_int32(k), _p(pruned),
+                              _p(sel), _p(fin))
+    return pruned[:n], sel[:n_seg, :k].reshape(n_seg, k), fin[:n_seg]

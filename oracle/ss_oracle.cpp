@@ -13,6 +13,9 @@
 //                             "LLM Inference and Serving" and "Experimental Setup").  The paper prints no
 //                             formula; this is the textbook definition, written per path with the path's
 //                             whole K/V materialised contiguously - no tiling, no sharing, no merging.
+//   ss_oracle_early_prune     The same selection while only part of the candidates is verified: rule 1 (ranked
+//                             below the top-k of the verified ones => pruned) and rule 2 (k perfect scores =>
+//                             final), paper, Section "Early Pruning of Search Tree".
 //   ss_oracle_topk            Selection of the top-k candidates by score (paper, Section "Early Pruning of
 //                             Search Tree": a candidate ranked below the top-k cannot be selected;
 //                             top-k = N / M).  Plain stable sort.
@@ -236,6 +239,54 @@ void ss_oracle_topk(const float* scores, const int32_t* seg_offsets, int32_t n_s
       } else {
         survivors[static_cast<int64_t>(s) * k + j] = -1;
       }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Early pruning during speculation (paper, Section "Early Pruning of Search Tree").  Only part of a problem's
+// candidates has been verified so far (verified[i] != 0; the scores of the others are ignored).  Per segment:
+//   rule 2  if at least k verified candidates have the perfect score (>= 1.0): the first k of them by index are
+//           selected, the segment is final, and every other candidate - verified or not - is pruned;
+//   rule 1  otherwise, if more than k candidates are verified: a verified candidate that ranks below the k best
+//           verified ones (score descending, lower index first among equals) cannot reach the final top-k and is
+//           pruned; unverified candidates keep running;
+//   if every candidate of the segment is verified the segment is final as well and the selection is the plain
+//   top-k.
+// pruned[i] = 1 iff candidate i must stop; selected = [P][k] indices (-1 padded; all -1 unless final);
+// final_out[s] = 1 iff segment s is final.
+// ---------------------------------------------------------------------------------------------------------
+void ss_oracle_early_prune(const float* scores, const uint8_t* verified, const int32_t* seg_offsets,
+                           int32_t n_segments, int32_t k, uint8_t* pruned, int32_t* selected, uint8_t* final_out) {
+  for (int32_t s = 0; s < n_segments; ++s) {
+    const int32_t lo = seg_offsets[s], hi = seg_offsets[s + 1];
+    for (int32_t j = 0; j < k; ++j) selected[static_cast<int64_t>(s) * k + j] = -1;
+    for (int32_t i = lo; i < hi; ++i) pruned[i] = 0;
+    final_out[s] = 0;
+    std::vector<int32_t> ver, perfect;
+    for (int32_t i = lo; i < hi; ++i) {
+      if (!verified[i]) continue;
+      ver.push_back(i);
+      if (scores[i] >= 1.0f) perfect.push_back(i);
+    }
+    if (static_cast<int32_t>(perfect.size()) >= k) {
+      for (int32_t i = lo; i < hi; ++i) pruned[i] = 1;
+      for (int32_t j = 0; j < k; ++j) {
+        selected[static_cast<int64_t>(s) * k + j] = perfect[j];
+        pruned[perfect[j]] = 0;
+      }
+      final_out[s] = 1;
+      continue;
+    }
+    std::stable_sort(ver.begin(), ver.end(),
+                     [scores](int32_t x, int32_t y) { return score_before(scores[x], scores[y]); });
+    const bool all_verified = static_cast<int32_t>(ver.size()) == hi - lo;
+    if (static_cast<int32_t>(ver.size()) > k)
+      for (size_t r = k; r < ver.size(); ++r) pruned[ver[r]] = 1;
+    if (all_verified) {
+      final_out[s] = 1;
+      for (int32_t j = 0; j < k && j < static_cast<int32_t>(ver.size()); ++j)
+        selected[static_cast<int64_t>(s) * k + j] = ver[j];
     }
   }
 }

@@ -485,3 +485,86 @@ def test_generator_shapes_config2_small():
         below = [p for p in range(w.num_paths) if n in w.chain(int(w.path_leaf_node[p]))]
         if below:
             assert below == list(range(below[0], below[-1] + 1))
+
+
+# =========================================================================================================
+# early pruning with partially verified candidates
+# =========================================================================================================
+def brute_early_prune(scores, verified, seg, k):
+    n = len(scores)
+    pruned = np.zeros(n, np.uint8)
+    sel = np.full((len(seg) - 1, k), -1, np.int32)
+    fin = np.zeros(len(seg) - 1, np.uint8)
+    for s in range(len(seg) - 1):
+        idx = list(range(seg[s], seg[s + 1]))
+        ver = [i for i in idx if verified[i]]
+        perfect = [i for i in ver if scores[i] >= 1.0]
+        if len(perfect) >= k:
+            chosen = perfect[:k]
+            for i in idx:
+                pruned[i] = 0 if i in chosen else 1
+            sel[s, :k] = chosen
+            fin[s] = 1
+            continue
+        order = sorted(ver, key=lambda i: (1 if math.isnan(scores[i]) else 0,
+                                           0.0 if math.isnan(scores[i]) else -(float(scores[i]) + 0.0), i))
+        if len(ver) > k:
+            for i in order[k:]:
+                pruned[i] = 1
+        if len(ver) == len(idx):
+            fin[s] = 1
+            sel[s, :min(k, len(order))] = order[:k]
+    return pruned, sel, fin
+
+
+def test_early_prune_paper_worked_example():
+    """The figure's walk-through: k = 1; B verified -> continues; D verified lower -> pruned; C perfect -> all others
+    pruned and C selected."""
+    lines = [l.strip() for l in open(os.path.join(GOLDEN, "early_pruning_example.txt")) if l.strip() and not l.startswith("#")]
+    k = int(lines[0].split()[1])
+    names = lines[1].split()[1:]
+    scores = np.zeros(len(names), np.float32)
+    verified = np.zeros(len(names), np.uint8)
+    seg = np.asarray([0, len(names)], np.int32)
+    cumulative_pruned = set()
+    for line in lines[2:]:
+        ev, pr, se = [x.strip() for x in line.split("|")]
+        _, who, val = ev.split()
+        scores[names.index(who)] = float(val)
+        verified[names.index(who)] = 1
+        pruned, sel, fin = oracle.early_prune(scores, verified, seg, k)
+        cumulative_pruned |= {names[i] for i in range(len(names)) if pruned[i]}
+        want_pruned = set() if pr.split(":")[1].strip() == "-" else set(pr.split(":")[1].split())
+        assert cumulative_pruned == want_pruned, line
+        want_sel = se.split(":")[1].strip()
+        if want_sel == "-":
+            assert fin[0] == 0 and list(sel[0]) == [-1] * k
+        else:
+            assert fin[0] == 1 and [names[i] for i in sel[0]] == want_sel.split()
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_early_prune_bruteforce_and_topk_consistency(seed):
+    rng = np.random.default_rng(400 + seed)
+    sizes = rng.integers(0, 30, size=7)
+    seg = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int32)
+    n = int(seg[-1])
+    sc = (rng.integers(0, 9, size=n) / 8.0).astype(np.float32)
+    sc[rng.random(n) < 0.25] = 1.0
+    k = int(rng.integers(1, 6))
+    for frac in (0.0, 0.3, 0.7, 1.0):
+        ver = (rng.random(n) < frac).astype(np.uint8) if frac < 1.0 else np.ones(n, np.uint8)
+        pruned, sel, fin = oracle.early_prune(sc, ver, seg, k)
+        bp, bs, bf = brute_early_prune(sc, ver, seg, k)
+        assert np.array_equal(pruned, bp) and np.array_equal(sel, bs) and np.array_equal(fin, bf)
+        # an unverified candidate is only ever pruned by rule 2 (segment final through perfect scores)
+        for s in range(len(sizes)):
+            for i in range(seg[s], seg[s + 1]):
+                if pruned[i] and not ver[i]:
+                    assert fin[s] == 1
+    # everything verified and fewer than k perfect scores in a segment => same survivors as the plain top-k
+    ver = np.ones(n, np.uint8)
+    sc2 = np.minimum(sc, np.float32(0.875))
+    pruned, sel, fin = oracle.early_prune(sc2, ver, seg, k)
+    surv, keep = oracle.topk(sc2, seg, k)
+    assert np.array_equal(1 - pruned, keep) and np.array_equal(sel, surv) and fin.all()
