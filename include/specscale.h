@@ -227,6 +227,31 @@ int32_t ss_topk_prune(const float* scores, const int32_t* seg_offsets, int32_t n
                       size_t workspace_bytes, void* stream);
 
 /* =========================================================================================================
+ * ss_early_prune - pruning while only part of a problem's candidates has been verified.
+ *
+ * Paper: Section "Early Pruning of Search Tree".  Rule 1: once more than k candidates are verified, a verified
+ * candidate ranked below the k best verified ones can no longer reach the final top-k and is pruned.  Rule 2: PRM
+ * scores lie in [0, 1]; once k verified candidates have the perfect score (>= 1.0) they are final - the first k of
+ * them by index are selected and every other candidate of the problem, verified or not, is pruned.  Worked example
+ * of the paper (k = 1): B verified -> continues; D verified with a lower score -> pruned; C perfect -> A, B, D
+ * pruned, C selected.  Ordering and special values as in ss_topk_prune.
+ *
+ *   scores        fp32 [n_total]    only entries with verified[i] != 0 are read
+ *   verified      uint8 [n_total]
+ *   seg_offsets   int32 [n_segments+1]; k host >= 1
+ *   pruned_out    uint8 [n_total]   1 iff the candidate must stop (entries outside every segment: 0)
+ *   selected_out  int32 [n_segments][k]  the selection of a FINAL segment (best first / perfect ones by index),
+ *                 -1 padded; all -1 while the segment is not final
+ *   final_out     uint8 [n_segments] 1 iff rule 2 fired or every candidate of the segment is verified (then
+ *                 selected_out equals the survivors of ss_topk_prune)
+ *   workspace     >= ss_topk_workspace_bytes(n_total) bytes, 256-byte aligned
+ * Errors: SS_ERR_INVALID_ARG, SS_ERR_WORKSPACE_TOO_SMALL, SS_ERR_CUDA.
+ * ======================================================================================================= */
+int32_t ss_early_prune(const float* scores, const uint8_t* verified, const int32_t* seg_offsets, int32_t n_segments,
+                       int32_t n_total, int32_t k, uint8_t* pruned_out, int32_t* selected_out, uint8_t* final_out,
+                       void* workspace, size_t workspace_bytes, void* stream);
+
+/* =========================================================================================================
  * Diagnostics
  * ======================================================================================================= */
 /* Number of kernels this library has launched in this process since it was loaded (host counter). */

@@ -34,7 +34,7 @@ EXPORTS = [
     "ss_status_string", "ss_last_device_status", "ss_dedup_workspace_bytes", "ss_dedup_paths",
     "ss_tree_attention_workspace_bytes", "ss_tree_attention", "ss_topk_workspace_bytes", "ss_topk_prune",
     "ss_launch_count", "ss_debug_umma_tile", "ss_profile_enable", "ss_profile_read",
-    "ss_dedup_paths_static", "ss_debug_tile_kernel_occupancy",
+    "ss_dedup_paths_static", "ss_debug_tile_kernel_occupancy", "ss_early_prune",
 ]
 PHASES = ["plan", "tiles", "leaves", "generic", "merge"]
 
@@ -225,6 +225,17 @@ def ss_topk_prune(scores, seg_offsets, n_segments, n_total, k, survivors_out, ke
                              ctypes.c_size_t(workspace.numel() if workspace is not None else 0), _stream(stream))
     if check:
         _check(rc, "ss_topk_prune")
+    return rc
+
+
+def ss_early_prune(scores, verified, seg_offsets, n_segments, n_total, k, pruned_out, selected_out, final_out,
+                   workspace, stream=None, check=True) -> int:
+    rc = lib().ss_early_prune(_ptr(scores), _ptr(verified), _ptr(seg_offsets), ctypes.c_int32(n_segments),
+                              ctypes.c_int32(n_total), ctypes.c_int32(k), _ptr(pruned_out), _ptr(selected_out),
+                              _ptr(final_out), _ptr(workspace),
+                              ctypes.c_size_t(workspace.numel() if workspace is not None else 0), _stream(stream))
+    if check:
+        _check(rc, "ss_early_prune")
     return rc
 
 

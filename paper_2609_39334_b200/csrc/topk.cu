@@ -67,8 +67,100 @@ topk_kernel(const float* __restrict__ scores, const int32_t* __restrict__ seg_of
   for (int j = n + threadIdx.x; j < k; j += blockDim.x) survivors[static_cast<int64_t>(s) * k + j] = -1;
 }
 
+// Early pruning with partially verified candidates (paper, Section "Early Pruning of Search Tree").  Same sort as
+// above over the VERIFIED candidates only (the others get the padding key and sort last); then
+//   rule 2: >= k verified candidates with the perfect score  -> the first k of them by index are selected, every
+//           other candidate of the segment is pruned, the segment is final;
+//   rule 1: more than k verified -> the verified candidates ranked below the k best are pruned;
+//   all verified -> final, selected = the k best.
+__global__ void __launch_bounds__(kThreads)
+early_prune_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ verified,
+                   const int32_t* __restrict__ seg_offsets, int k, uint8_t* __restrict__ pruned,
+                   int32_t* __restrict__ selected, uint8_t* __restrict__ final_out, uint64_t* __restrict__ scratch) {
+  __shared__ uint64_t smem_keys[kSmemKeys];
+  __shared__ int s_nver, s_nperfect;
+  const int s = blockIdx.x;
+  const int lo = seg_offsets[s], hi = seg_offsets[s + 1];
+  const int n = hi - lo;
+  for (int j = threadIdx.x; j < k; j += blockDim.x) selected[static_cast<int64_t>(s) * k + j] = -1;
+  if (n <= 0) {
+    if (threadIdx.x == 0) final_out[s] = 1;      // nothing left to verify in an empty segment
+    return;
+  }
+  if (threadIdx.x == 0) { s_nver = 0; s_nperfect = 0; }
+  __syncthreads();
+  int n_pad = 1;
+  while (n_pad < n) n_pad <<= 1;
+  uint64_t* keys = (n_pad <= kSmemKeys) ? smem_keys : (scratch + 2 * static_cast<int64_t>(lo));
+  int my_ver = 0, my_perfect = 0;
+  for (int i = threadIdx.x; i < n_pad; i += blockDim.x) {
+    uint64_t key = ~0ull;
+    if (i < n && verified[lo + i]) {
+      const float f = scores[lo + i];
+      key = make_key(f, static_cast<uint32_t>(i));
+      ++my_ver;
+      if (f >= 1.0f) ++my_perfect;
+    }
+    keys[i] = key;
+  }
+  if (my_ver) atomicAdd(&s_nver, my_ver);
+  if (my_perfect) atomicAdd(&s_nperfect, my_perfect);
+  __syncthreads();
+  const int nver = s_nver, nperfect = s_nperfect;
+  if (nperfect >= k) {
+    // rule 2: rank of a perfect candidate among the perfect ones by index (segments are small: a counting loop)
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+      bool chosen = false;
+      if (verified[lo + i] && scores[lo + i] >= 1.0f) {
+        int before = 0;
+        for (int j = 0; j < i; ++j) before += (verified[lo + j] && scores[lo + j] >= 1.0f) ? 1 : 0;
+        if (before < k) {
+          chosen = true;
+          selected[static_cast<int64_t>(s) * k + before] = lo + i;
+        }
+      }
+      pruned[lo + i] = chosen ? 0 : 1;
+    }
+    if (threadIdx.x == 0) final_out[s] = 1;
+    return;
+  }
+  bitonic_sort(keys, n_pad);
+  const bool all_verified = nver == n;
+  for (int i = threadIdx.x; i < n; i += blockDim.x)
+    if (!verified[lo + i]) pruned[lo + i] = 0;
+  for (int j = threadIdx.x; j < nver; j += blockDim.x) {
+    const int cand = lo + static_cast<int>(keys[j] & 0xffffffffu);
+    pruned[cand] = (nver > k && j >= k) ? 1 : 0;
+    if (all_verified && j < k) selected[static_cast<int64_t>(s) * k + j] = cand;
+  }
+  if (threadIdx.x == 0) final_out[s] = all_verified ? 1 : 0;
+}
+
 }  // namespace topk
 }  // namespace ss
+
+extern "C" int32_t ss_early_prune(const float* scores, const uint8_t* verified, const int32_t* seg_offsets,
+                                  int32_t n_segments, int32_t n_total, int32_t k, uint8_t* pruned_out,
+                                  int32_t* selected_out, uint8_t* final_out, void* workspace, size_t workspace_bytes,
+                                  void* stream) {
+  using namespace ss;
+  if (n_segments < 0 || n_total < 0 || k < 1) return SS_ERR_INVALID_ARG;
+  cudaStream_t st = as_stream(stream);
+  if (n_total > 0 && pruned_out && cudaMemsetAsync(pruned_out, 0, static_cast<size_t>(n_total), st) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return SS_ERR_CUDA;
+  }
+  if (n_segments == 0) return SS_OK;
+  if (!seg_offsets || !selected_out || !final_out || !workspace) return SS_ERR_INVALID_ARG;
+  if (n_total > 0 && (!scores || !verified || !pruned_out)) return SS_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return SS_ERR_INVALID_ARG;
+  size_t need = 0;
+  ss_topk_workspace_bytes(n_total, &need);
+  if (workspace_bytes < need) return SS_ERR_WORKSPACE_TOO_SMALL;
+  SS_LAUNCH(topk::early_prune_kernel, n_segments, topk::kThreads, 0, st, scores, verified, seg_offsets, k, pruned_out,
+            selected_out, final_out, static_cast<uint64_t*>(workspace));
+  return SS_OK;
+}
 
 extern "C" int32_t ss_topk_workspace_bytes(int32_t n_total, size_t* out_bytes) {
   if (n_total < 0 || !out_bytes) return SS_ERR_INVALID_ARG;
