@@ -157,7 +157,7 @@ def oracle_sample(w, seed=0):
     return np.asarray(sorted(chosen), np.int64)
 
 
-def time_oracle(w_host, sample, steps, warmup):
+def time_oracle(w_host, steps, warmup):
     import oracle
     times = []
     for it in range(warmup + steps):
@@ -208,7 +208,7 @@ def main():
         del w
         if dev != "cpu":
             torch.cuda.empty_cache()
-        sec = time_oracle(sub, sample, max(args.steps, 1), min(args.warmup, 1))
+        sec = time_oracle(sub, max(args.steps, 1), min(args.warmup, 1))
         tokens = int(sub.path_q_len.astype(np.int64).sum())
         val = tokens / sec
         what = (f"{len(sample)} unique paths of {args.workload} ({int((sub.path_q_len > 1).sum())} verification, "
@@ -384,7 +384,7 @@ def main():
         oracle.build()
         sample = oracle_sample(w)
         sub = synth.extract_subworkload(w, sample)
-        sec = time_oracle(sub, sample, 1, 0)
+        sec = time_oracle(sub, 1, 0)
         stok = int(sub.path_q_len.astype(np.int64).sum())
         out["cpu_baseline"] = {
             "value": stok / sec, "unit": UNIT, "cores": oracle.host_cores(), "kind": "oracle",

@@ -7,7 +7,6 @@ library is missing, loading fails with an error.
 from __future__ import annotations
 
 import ctypes
-import math
 import os
 from typing import Optional
 

@@ -7,7 +7,7 @@ to the caller (after deduplication a sequence has a single query row, so Q exist
 """
 from __future__ import annotations
 
-from typing import Dict, Optional
+from typing import Dict
 
 import numpy as np
 import torch
