@@ -152,7 +152,8 @@ int32_t ss_dedup_paths_static(const int32_t* tok_ids, const int64_t* tok_offsets
  * rows of 256 bytes), kv_page_stride and kv_head_stride multiples of 128 elements, k_pool and v_pool 256-byte
  * aligned.  The recommended pool is one allocation laid out [page][K|V][kv head][16][128].
  *
- * q   bf16 [total_q][Hq][128], rows of path p are q_offsets[p] .. q_offsets[p+1]-1, 16-byte aligned
+ * q   bf16 [total_q][Hq][128], rows of path p are q_offsets[p] .. q_offsets[p+1]-1 (or start at q_src_offsets[p] in
+ *     a larger array, see the descriptor), 16-byte aligned
  * out bf16 [total_q][Hq][128]   (fp32 accumulation, rounded to nearest even), 16-byte aligned
  * lse fp32 [total_q][Hq]        or NULL
  *
@@ -194,6 +195,12 @@ typedef struct ss_attn_desc {
   /* ---- sizing hints (host scalars; 0 = use the safe default; tight values shrink the workspace) ---- */
   int32_t max_depth;                 /* nodes on the longest chain; default SS_MAX_DEPTH */
   int32_t max_decode_paths;          /* paths with T == 1; default num_paths */
+  /* ---- optional query indirection ---- */
+  const int64_t* q_src_offsets;      /* NULL, or [num_paths]: row of q where path p's T query rows start (default
+                                        q_offsets[p]).  Lets the caller leave q in logical-candidate order after
+                                        ss_dedup_paths instead of gathering the unique paths' rows; out / lse rows
+                                        stay at q_offsets[p] */
+  int64_t q_src_rows;                /* rows addressable through q when q_src_offsets is given (host) */
   /* ---- data ---- */
   const void* q;
   void* out;

@@ -61,6 +61,7 @@ class ss_attn_desc_t(ctypes.Structure):
         ("num_paths_dev", ctypes.c_void_p), ("path_leaf_node", ctypes.c_void_p), ("path_q_len", ctypes.c_void_p),
         ("q_offsets", ctypes.c_void_p), ("total_q", ctypes.c_int64),
         ("max_depth", ctypes.c_int32), ("max_decode_paths", ctypes.c_int32),
+        ("q_src_offsets", ctypes.c_void_p), ("q_src_rows", ctypes.c_int64),
         ("q", ctypes.c_void_p), ("out", ctypes.c_void_p), ("lse", ctypes.c_void_p),
     ]
 
@@ -161,7 +162,7 @@ def make_attn_desc(*, num_q_heads, num_kv_heads, kv_pool=None, k_pool=None, v_po
                    kv_page_stride=None, kv_head_stride=None, kv_token_stride=None, node_parent, node_kv_len,
                    node_page_offsets, node_pages, total_node_pages, path_leaf_node, path_q_len, q_offsets, total_q,
                    q, out, lse=None, num_paths=None, num_paths_dev=None, sm_scale=0.0, flags=0, max_depth=0,
-                   max_decode_paths=0, head_dim=128, page_size=16) -> ss_attn_desc_t:
+                   max_decode_paths=0, head_dim=128, page_size=16, q_src_offsets=None, q_src_rows=0) -> ss_attn_desc_t:
     """Fills the descriptor.  `kv_pool` is the recommended single allocation [page][2][Hkv][16][128]; otherwise
     give k_pool / v_pool tensors and the element strides."""
     d = ss_attn_desc_t()
@@ -189,6 +190,8 @@ def make_attn_desc(*, num_q_heads, num_kv_heads, kv_pool=None, k_pool=None, v_po
     d.path_leaf_node, d.path_q_len, d.q_offsets = path_leaf_node.data_ptr(), path_q_len.data_ptr(), q_offsets.data_ptr()
     d.total_q = int(total_q)
     d.max_depth, d.max_decode_paths = int(max_depth), int(max_decode_paths)
+    d.q_src_offsets = q_src_offsets.data_ptr() if q_src_offsets is not None else None
+    d.q_src_rows = int(q_src_rows)
     d.q = q.data_ptr() if q is not None else None
     d.out = out.data_ptr() if out is not None else None
     d.lse = lse.data_ptr() if lse is not None else None

@@ -102,6 +102,7 @@ static Layout carve(const ss_attn_desc_t* d, char* base, Params* P) {
   char* path_arrays[6];
   for (int i = 0; i < 6; ++i) path_arrays[i] = take(NP * 4);
   char* dec_tok = take((static_cast<size_t>(cap_dec) + 1) * 4);
+  char* dec_src = take((static_cast<size_t>(cap_dec) + 1) * 4);
   char* dec_slot = take((static_cast<size_t>(cap_dec) + 1) * 4);
   char* tiles = take(static_cast<size_t>(caps.tile_items) * sizeof(TileItem));
   char* leaves = take(static_cast<size_t>(caps.leaf_items) * sizeof(LeafItem));
@@ -116,6 +117,7 @@ static Layout carve(const ss_attn_desc_t* d, char* base, Params* P) {
                        &P->path_chain_base};
     for (int i = 0; i < 6; ++i) *pp[i] = reinterpret_cast<int32_t*>(path_arrays[i]);
     P->dec_tok = reinterpret_cast<int32_t*>(dec_tok);
+    P->dec_src = reinterpret_cast<int32_t*>(dec_src);
     P->dec_slot_base = reinterpret_cast<int32_t*>(dec_slot);
     P->tile_items = reinterpret_cast<TileItem*>(tiles);
     P->leaf_items = reinterpret_cast<LeafItem*>(leaves);
@@ -156,6 +158,7 @@ extern "C" int32_t ss_tree_attention(const ss_attn_desc_t* d, void* workspace, s
       reinterpret_cast<uintptr_t>(d->q) % 16 || reinterpret_cast<uintptr_t>(d->out) % 16)
     return SS_ERR_UNSUPPORTED;
   if (d->total_q > 0x7fffffffLL / d->num_q_heads) return SS_ERR_UNSUPPORTED;   // row indices are int32
+  if (d->q_src_offsets && (d->q_src_rows < 0 || d->q_src_rows > 0x7fffffffLL / d->num_q_heads)) return SS_ERR_INVALID_ARG;
 
   Params P;
   memset(&P, 0, sizeof P);
@@ -185,6 +188,8 @@ extern "C" int32_t ss_tree_attention(const ss_attn_desc_t* d, void* workspace, s
   P.path_leaf_node = d->path_leaf_node;
   P.path_q_len = d->path_q_len;
   P.q_offsets = d->q_offsets;
+  P.q_src_offsets = d->q_src_offsets;
+  P.q_src_rows = d->q_src_rows;
   P.total_q = d->total_q;
   P.q = static_cast<const __nv_bfloat16*>(d->q);
   P.out = static_cast<__nv_bfloat16*>(d->out);

@@ -60,7 +60,7 @@ __global__ void __launch_bounds__(kLeafWarps * 32) leaf_items_kernel(const Param
     // ---- query fragments (dim-permuted, see above) --------------------------------------------------------
     uint4 qa[4], qb[4];
     {
-      const __nv_bfloat16* q0 = P.q + (static_cast<int64_t>(it.q_row) * P.Hq + it.g * G) * kHeadDim;
+      const __nv_bfloat16* q0 = P.q + (static_cast<int64_t>(it.q_src) * P.Hq + it.g * G) * kHeadDim;
 #pragma unroll
       for (int k2 = 0; k2 < 4; ++k2) {
         qa[k2] = gid < G ? ldg128(q0 + gid * kHeadDim + 32 * k2 + 8 * tig) : make_uint4(0, 0, 0, 0);

@@ -126,8 +126,13 @@ __global__ void __launch_bounds__(kGridThreads) plan_paths_kernel(const Params P
     const int p = static_cast<int>(p64);
     const int leaf = P.path_leaf_node[p];
     const int T = P.path_q_len[p];
+    bool bad_src = false;
+    if (P.q_src_offsets) {
+      const int64_t s0 = P.q_src_offsets[p];
+      bad_src = s0 < 0 || s0 + T > P.q_src_rows || s0 + T > 0x7fffffffLL;
+    }
     if (leaf < 0 || leaf >= N || T < 1 || P.q_offsets[p + 1] - P.q_offsets[p] != T || P.q_offsets[p] < 0 ||
-        P.q_offsets[p + 1] > P.total_q) {
+        P.q_offsets[p + 1] > P.total_q || bad_src) {
       set_status(&hdr->status, SS_ERR_BAD_INPUT);
       P.path_class[p] = kClassGeneric;
       continue;
@@ -271,7 +276,9 @@ __global__ void __launch_bounds__(kGridThreads) plan_emit_kernel(const Params P)
       const int rank = P.path_dec_rank[p];
       const int leaf = P.path_leaf_node[p];
       const int len = P.node_kv_len[leaf];
+      const int32_t src_row = static_cast<int32_t>(P.q_src_offsets ? P.q_src_offsets[p] : P.q_offsets[p]);
       P.dec_tok[rank] = static_cast<int32_t>(P.q_offsets[p]);
+      P.dec_src[rank] = src_row;
       P.dec_slot_base[rank] = P.path_slot_base[p];
       if (!(P.node_npaths[leaf] == 1 && len > 0)) continue;
       const int chunks = ceil_div(len, kLeafChunk);
@@ -286,13 +293,15 @@ __global__ void __launch_bounds__(kGridThreads) plan_emit_kernel(const Params P)
           it.kv_begin = c * kLeafChunk;
           it.kv_end = min(len, (c + 1) * kLeafChunk);
           it.slot = slot0 + c;
-          it.pad0 = it.pad1 = 0;
+          it.q_src = src_row;
+          it.pad1 = 0;
           P.leaf_items[e++] = it;
         }
     } else if (cls == kClassChain) {
       const int T = P.path_q_len[p];
       const int L = P.path_kv_len[p];
       const int tiles = ceil_div(T, tpt);
+      const int32_t src_row = static_cast<int32_t>(P.q_src_offsets ? P.q_src_offsets[p] : P.q_offsets[p]);
       int e = n_stacked + P.path_chain_base[p];
       for (int g = 0; g < P.Hkv; ++g)
         for (int t = 0; t < tiles; ++t) {
@@ -305,6 +314,8 @@ __global__ void __launch_bounds__(kGridThreads) plan_emit_kernel(const Params P)
           it.limit0 = L - T + t * tpt + 1;
           it.kv_end = max(0, min(L, it.limit0 + it.n_tok - 1));
           it.slot_off = -1;
+          it.src0 = src_row + t * tpt;
+          it.pad = 0;
           P.tile_items[e++] = it;
         }
     }
@@ -337,6 +348,8 @@ __global__ void __launch_bounds__(kGridThreads) plan_emit_kernel(const Params P)
     it.kv_end = min(len, (split + 1) * split_len);
     it.limit0 = it.kv_end;
     it.slot_off = P.node_level_off[n] + split;
+    it.src0 = 0;
+    it.pad = 0;
     P.tile_items[e] = it;
   }
 }

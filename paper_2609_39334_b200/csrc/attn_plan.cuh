@@ -27,7 +27,7 @@ constexpr int kMinSplitLen = 512;       // a split is at least this many keys
 enum PathClass : int32_t { kClassDecode = 0, kClassChain = 1, kClassGeneric = 2 };
 enum ItemKind : int32_t { kItemStacked = 0, kItemChain = 1 };
 
-// One tile of stacked query rows against a KV source.  32 bytes.
+// One tile of stacked query rows against a KV source.  40 bytes.
 struct TileItem {
   int32_t node;       // stacked: the shared node; chain: the path's leaf node
   int32_t tok0;       // stacked: index into dec_tok[]; chain: first query row (global token index)
@@ -37,6 +37,8 @@ struct TileItem {
   int32_t kv_end;
   int32_t limit0;     // keys visible to the tile's first token; token i sees limit0 + i * (kind == chain)
   int32_t slot_off;   // stacked: partial slot relative to the token's slot base; chain: -1 (final output)
+  int32_t src0;       // chain: row of q holding the tile's first token (stacked: rows come from dec_src[])
+  int32_t pad;
 };
 
 // One chunk of a decode path's private leaf.  32 bytes.
@@ -47,7 +49,8 @@ struct LeafItem {
   int32_t kv_begin;   // token range inside the leaf
   int32_t kv_end;
   int32_t slot;       // absolute partial slot
-  int32_t pad0, pad1;
+  int32_t q_src;      // row of q holding the token's query
+  int32_t pad1;
 };
 
 struct PlanHeader {       // first bytes of the workspace; status MUST be the first word
@@ -84,6 +87,8 @@ struct Params {
   int32_t num_paths;
   const int32_t *num_paths_dev, *path_leaf_node, *path_q_len;
   const int64_t* q_offsets;
+  const int64_t* q_src_offsets;  // optional: where each path's query rows start inside q
+  int64_t q_src_rows;
   int64_t total_q;
   const __nv_bfloat16* q;
   __nv_bfloat16* out;
@@ -95,7 +100,7 @@ struct Params {
   int32_t *node_start, *node_depth, *node_first, *node_last, *node_npaths, *node_ndec, *node_own_slots,
       *node_level_off, *node_item_base, *node_splits, *node_split_len;
   int32_t *path_class, *path_kv_len, *path_dec_rank, *path_slot_base, *path_leaf_base, *path_chain_base;
-  int32_t *dec_tok, *dec_slot_base;
+  int32_t *dec_tok, *dec_src, *dec_slot_base;   // per decode token: output row, query row, first partial slot
   TileItem* tile_items;
   LeafItem* leaf_items;
   float* part_o;             // [slots][Hq][128]

@@ -109,7 +109,8 @@ __global__ void generic_kernel(const Params P) {
     const int t = static_cast<int>(q_row - P.q_offsets[p]);
     const int visible = P.path_kv_len[p] - T + t + 1;
     RowState r;
-    row_init(r, P.q + (q_row * P.Hq + h) * kHeadDim, lane);
+    const int64_t q_src = P.q_src_offsets ? P.q_src_offsets[p] + t : q_row;
+    row_init(r, P.q + (q_src * P.Hq + h) * kHeadDim, lane);
     if (visible > 0) row_visit_chain(r, P, P.path_leaf_node[p], h / P.G, 0, visible, lane);
     row_store_final(r, P, q_row, h, lane);
   }
@@ -127,10 +128,11 @@ __global__ void tile_items_simple(const Params P) {
       const int i = rrow / P.G, h = g * P.G + rrow % P.G;
       const int dec = it.tok0 + i;                       // stacked: index into dec_tok
       const int64_t q_row = (kind == kItemChain) ? static_cast<int64_t>(it.tok0 + i) : P.dec_tok[dec];
+      const int64_t q_src = (kind == kItemChain) ? static_cast<int64_t>(it.src0 + i) : P.dec_src[dec];
       const int visible = (kind == kItemChain) ? it.limit0 + i : it.limit0;
       const int v1 = min(it.kv_end, visible);
       RowState r;
-      row_init(r, P.q + (q_row * P.Hq + h) * kHeadDim, lane);
+      row_init(r, P.q + (q_src * P.Hq + h) * kHeadDim, lane);
       if (kind == kItemChain) {
         row_visit_chain(r, P, it.node, g, it.kv_begin, v1, lane);
         row_store_final(r, P, q_row, h, lane);
@@ -151,7 +153,7 @@ __global__ void leaf_items_simple(const Params P) {
     const LeafItem it = P.leaf_items[w / P.G];
     const int h = it.g * P.G + static_cast<int>(w % P.G);
     RowState r;
-    row_init(r, P.q + (static_cast<int64_t>(it.q_row) * P.Hq + h) * kHeadDim, lane);
+    row_init(r, P.q + (static_cast<int64_t>(it.q_src) * P.Hq + h) * kHeadDim, lane);
     row_visit_node(r, P, it.node, it.g, it.kv_begin, it.kv_end, lane);
     row_store_partial(r, P, it.slot, h, lane);
   }

@@ -60,7 +60,7 @@ __device__ __forceinline__ float ex2(float x) {
 }
 
 struct ItemView {
-  int node, tok0, n_tok, kind, g, kv_begin, kv_end, limit0, slot_off, n_tiles;
+  int node, tok0, n_tok, kind, g, kv_begin, kv_end, limit0, slot_off, src0, n_tiles;
 };
 
 __device__ __forceinline__ ItemView view(const TileItem& it) {
@@ -68,6 +68,7 @@ __device__ __forceinline__ ItemView view(const TileItem& it) {
   v.node = it.node; v.tok0 = it.tok0; v.n_tok = it.n_tok;
   v.kind = it.kind_g >> 16; v.g = it.kind_g & 0xffff;
   v.kv_begin = it.kv_begin; v.kv_end = it.kv_end; v.limit0 = it.limit0; v.slot_off = it.slot_off;
+  v.src0 = it.src0;
   v.n_tiles = v.kv_end > v.kv_begin ? (v.kv_end - v.kv_begin + kKvTile - 1) / kKvTile : 0;
   return v;
 }
@@ -125,11 +126,11 @@ tile_items_umma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_
       const int i = row / G, hl = row - i * G;
       const bool row_valid = i < it.n_tok;
       const int h = it.g * G + hl;
-      int64_t q_row = 0;
+      int64_t q_row = 0, q_src = 0;                               // output row / row of q holding the query
       int dec = 0;
       if (row_valid) {
-        if (it.kind == kItemChain) q_row = it.tok0 + i;
-        else { dec = it.tok0 + i; q_row = P.dec_tok[dec]; }
+        if (it.kind == kItemChain) { q_row = it.tok0 + i; q_src = it.src0 + i; }
+        else { dec = it.tok0 + i; q_row = P.dec_tok[dec]; q_src = P.dec_src[dec]; }
       }
       const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
       float m = -INFINITY, l = 0.f;
@@ -137,7 +138,7 @@ tile_items_umma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_
       if (n_tiles > 0) {
         // ---- Q rows into the UMMA operand layout ---------------------------------------------------------------
         {
-          const uint4* src = reinterpret_cast<const uint4*>(P.q + (q_row * P.Hq + h) * kHeadDim);
+          const uint4* src = reinterpret_cast<const uint4*>(P.q + (q_src * P.Hq + h) * kHeadDim);
 #pragma unroll
           for (int ch = 0; ch < 16; ++ch) {
             const uint4 v = row_valid ? __ldg(src + ch) : make_uint4(0, 0, 0, 0);

@@ -2,8 +2,8 @@
 workspace tensors, and runs   ss_dedup_paths -> (gather of the unique paths) -> ss_tree_attention -> ss_topk_prune.
 
 Only memory management and argument marshalling happen here.  The one data movement that is not a library call is
-the compaction of the per-path descriptor arrays and query rows by `unique_paths` - a plain gather that belongs
-to the caller (after deduplication a sequence has a single query row, so Q exists only for unique paths).
+the compaction of the small per-path descriptor arrays by `unique_paths` - a plain gather that belongs to the
+caller.  The query rows themselves are not moved: the attention call reads them in place through `q_src_offsets`.
 """
 from __future__ import annotations
 
@@ -65,17 +65,17 @@ class DevicePipeline:
         self.u_q_len = torch.empty(max(N, 1), **i32)
         self.u_q_offsets = torch.zeros(N + 1, dtype=torch.int64, device=dev)
         total_q = w.total_q
-        self.u_q = torch.empty((max(total_q, 1), w.num_q_heads, w.head_dim), dtype=torch.bfloat16, device=dev)
-        self.out = torch.empty_like(self.u_q)
+        self.u_q_src = torch.zeros(max(N, 1), dtype=torch.int64, device=dev)
+        self.out = torch.empty((max(total_q, 1), w.num_q_heads, w.head_dim), dtype=torch.bfloat16, device=dev)
         self.lse = torch.empty((max(total_q, 1), w.num_q_heads), dtype=torch.float32, device=dev)
-        self.q_row_of = torch.empty(max(total_q, 1), dtype=torch.int64, device=dev)
         depth = self._max_depth(w)
         self.desc = B.make_attn_desc(
             num_q_heads=w.num_q_heads, num_kv_heads=w.num_kv_heads, kv_pool=self.kv_pool,
             node_parent=self.node_parent, node_kv_len=self.node_kv_len, node_page_offsets=self.node_page_offsets,
             node_pages=self.node_pages, total_node_pages=int(w.node_page_offsets[-1]),
             path_leaf_node=self.u_leaf, path_q_len=self.u_q_len, q_offsets=self.u_q_offsets, total_q=total_q,
-            q=self.u_q, out=self.out, lse=self.lse, num_paths=N, num_paths_dev=self.num_unique,
+            q=self.q, q_src_offsets=self.u_q_src, q_src_rows=total_q, out=self.out, lse=self.lse, num_paths=N,
+            num_paths_dev=self.num_unique,
             sm_scale=sm_scale, flags=attn_flags, max_depth=depth,
             max_decode_paths=int((w.path_q_len == 1).sum()))
         self.attn_ws = B.alloc_workspace(B.ss_tree_attention_workspace_bytes(self.desc), dev)
@@ -100,8 +100,8 @@ class DevicePipeline:
                          self.num_unique, self.dedup_ws, stream=stream)
 
     def compact_unique(self):
-        """Gather of the unique paths' descriptor rows and query rows (device-side, no host sync: entries past
-        the live count U are computed from clamped indices and ignored by the attention call)."""
+        """Gather of the unique paths' descriptor rows (device-side, no host sync: entries past the live count U are
+        computed from clamped indices and ignored by the attention call).  Query rows stay where they are."""
         N = self.N
         if N == 0:
             return
@@ -113,15 +113,7 @@ class DevicePipeline:
         T = torch.where(live, self.path_q_len[src].long(), torch.zeros_like(ar))
         self.u_q_len[:N] = T.to(torch.int32)
         self.u_q_offsets[1:] = torch.cumsum(T, 0)
-        # query rows: row r of the compacted Q comes from row q_offsets[src[p]] + (r - u_q_offsets[p])
-        total = self.w.total_q
-        if total:
-            rows = torch.arange(total, device=self.device)
-            p = torch.searchsorted(self.u_q_offsets[1:], rows, right=True).clamp_(max=N - 1)
-            src_row = self.q_offsets[src[p]] + (rows - self.u_q_offsets[p])
-            src_row.clamp_(0, total - 1)
-            self.q_row_of[:total] = src_row
-            torch.index_select(self.q, 0, src_row, out=self.u_q[:total])
+        self.u_q_src[:N] = self.q_offsets[src]
 
     def attention(self, stream=None):
         B.ss_tree_attention(self.desc, self.attn_ws, stream=stream)

@@ -415,3 +415,33 @@ def test_config5_full_size_sampled_outputs():
     lerr = np.abs(lse - l_ref).max()
     assert err.max() <= OUT_MAX and err.mean() <= OUT_MEAN and lerr <= LSE_MAX, (err.max(), err.mean(), lerr)
     assert err.max() <= TIGHT_OUT_MAX and err.mean() <= TIGHT_OUT_MEAN and lerr <= TIGHT_LSE, (err.max(), err.mean(), lerr)
+
+
+def test_attention_without_query_indirection_matches():
+    """q_src_offsets = NULL (queries already compacted at q_offsets) gives the same result as reading them in place."""
+    w = synth.build_tree_workload("noind", 77, 12, 2, [128], [6], 2, (1, 120), lambda i, n, rng: 1 + (i % 2) * 30,
+                                  dup_frac=0.25)
+    pipe = DevicePipeline(w, DEV)
+    pipe.dedup()
+    pipe.compact_unique()
+    pipe.attention()
+    r = pipe.results()
+    U, tq = r["num_unique"], r["total_q"]
+    src = pipe.u_q_src[:U].cpu().numpy()
+    T = pipe.u_q_len[:U].cpu().numpy()
+    rows = np.concatenate([np.arange(s, s + t) for s, t in zip(src, T)])
+    q_compact = pipe.q[torch.from_numpy(rows).to(DEV)].contiguous()
+    out = torch.empty_like(q_compact)
+    lse = torch.empty((tq, w.num_q_heads), dtype=torch.float32, device=DEV)
+    desc = B.make_attn_desc(
+        num_q_heads=w.num_q_heads, num_kv_heads=w.num_kv_heads, kv_pool=pipe.kv_pool, node_parent=pipe.node_parent,
+        node_kv_len=pipe.node_kv_len, node_page_offsets=pipe.node_page_offsets, node_pages=pipe.node_pages,
+        total_node_pages=int(w.node_page_offsets[-1]), path_leaf_node=pipe.u_leaf[:U].contiguous(),
+        path_q_len=pipe.u_q_len[:U].contiguous(), q_offsets=pipe.u_q_offsets[:U + 1].contiguous(), total_q=tq,
+        q=q_compact, out=out, lse=lse)
+    ws = B.alloc_workspace(B.ss_tree_attention_workspace_bytes(desc), DEV)
+    B.ss_tree_attention(desc, ws)
+    torch.cuda.synchronize()
+    assert B.ss_last_device_status(ws) == B.SS_OK
+    assert np.array_equal(out.to(torch.float64).cpu().numpy(), r["out"])
+    assert np.array_equal(lse.to(torch.float64).cpu().numpy(), r["lse"])
