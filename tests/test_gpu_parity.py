@@ -445,3 +445,25 @@ def test_attention_without_query_indirection_matches():
     assert B.ss_last_device_status(ws) == B.SS_OK
     assert np.array_equal(out.to(torch.float64).cpu().numpy(), r["out"])
     assert np.array_equal(lse.to(torch.float64).cpu().numpy(), r["lse"])
+
+
+def test_attention_reports_too_small_workspace_from_the_device():
+    """Sizing hints that are too low are caught by the planner (status read back), nothing is written out of bounds."""
+    w = synth.build_tree_workload("hint", 9, 8, 2, [64], [12], 2, (1, 300), lambda i, n, rng: 1)
+    pipe = DevicePipeline(w, DEV)
+    pipe.dedup()
+    pipe.compact_unique()
+    good = B.ss_tree_attention_workspace_bytes(pipe.desc)
+    pipe.desc.max_decode_paths = 3                       # 24 decode paths exist
+    small = B.ss_tree_attention_workspace_bytes(pipe.desc)
+    assert small < good
+    canary = torch.full((4096,), 0x5A, dtype=torch.uint8, device=DEV)
+    ws_all = torch.cat([B.alloc_workspace(small, DEV)[:small + (-small) % 256], canary])
+    ws = ws_all[:ws_all.numel() - 4096]
+    B.ss_tree_attention(pipe.desc, ws)
+    torch.cuda.synchronize()
+    assert B.ss_last_device_status(ws) == B.SS_ERR_WORKSPACE_TOO_SMALL
+    assert bool((ws_all[-4096:] == 0x5A).all())         # nothing past the workspace was touched
+    # host-side check: a workspace smaller than the query result is refused before any launch
+    rc = B.ss_tree_attention(pipe.desc, ws[:1024], check=False)
+    assert rc == B.SS_ERR_WORKSPACE_TOO_SMALL
