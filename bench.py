@@ -28,6 +28,7 @@ if ROOT not in sys.path:
 METRIC = "candidate_path_query_tokens_per_s"
 UNIT = "tokens/s"
 WORKLOADS = {"c2": 2, "c3": 3, "c4": 4, "c5": 5}
+LV_SWEEP_TOKENS = [256, 512, 1024, 2048, 4096, 8192, 16384]
 L2_BYTES = 126 * 1024 * 1024
 
 
@@ -171,12 +172,59 @@ def time_oracle(w_host, steps, warmup):
 
 
 # ------------------------------------------------------------------------------------------------------------
+def lv_sweep(args):
+    """Attention-only analogue of the paper's verification-throughput profile (Section "Lazy Verification": the
+    token threshold of the first flush policy is read off a throughput-vs-batched-tokens curve).  For each batch
+    size a set of verification steps (7B reward-model head shape, 1024-token prompt, 64-512 prior tokens, steps of
+    16-128 tokens, 8 candidates per problem) is attended in one ss_tree_attention call; reported is step tokens/s."""
+    import torch
+    from paper_2609_39334_b200 import binding as B
+    from paper_2609_39334_b200 import synth
+    from paper_2609_39334_b200.pipeline import DevicePipeline
+    assert torch.cuda.is_available(), "bench.py needs a GPU (there is no CPU fallback)"
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=dev)
+    curve = []
+    for target in LV_SWEEP_TOKENS:
+        problems = max(1, target // (8 * 72))
+        per = max(1, round(target / (72 * problems)))
+        w = synth.build_tree_workload(f"lv{target}", synth.BASE_SEED + 100 + target, 28, 4, [1024], [per], problems,
+                                      (64, 512), lambda i, n, rng: int(rng.integers(16, 129)), device=dev)
+        pipe = DevicePipeline(w, dev)
+        pipe.dedup()
+        pipe.compact_unique()
+        for _ in range(max(args.warmup, 3)):
+            pipe.attention()
+        torch.cuda.synchronize(dev)
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+        for a, b in ev:
+            flush.fill_(1)
+            a.record()
+            pipe.attention()
+            b.record()
+        torch.cuda.synchronize(dev)
+        st = B.ss_last_device_status(pipe.attn_ws)
+        if st != B.SS_OK:
+            raise B.SpecScaleError(st, "lv-sweep")
+        ms = float(np.median([a.elapsed_time(b) for a, b in ev]))
+        tokens = int(w.path_q_len.sum())
+        curve.append({"batched_tokens": tokens, "candidates": w.num_paths, "ms": ms, "tokens_per_s": tokens / (ms * 1e-3)})
+    print(json.dumps({"metric": "verification_attention_step_tokens_per_s", "unit": "tokens/s", "n_gpus": 1,
+                      "steps": args.steps, "warmup": max(args.warmup, 3), "dtype": "bf16", "data": "synthetic",
+                      "config": {"workload": "lv-sweep", "heads": "28q/4kv", "prefix": 1024, "l2": "L2 flushed between iterations"},
+                      "curve": curve}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="c5", choices=sorted(WORKLOADS))
+    ap.add_argument("--workload", default="c5", choices=sorted(WORKLOADS) + ["lv-sweep"],
+                    help="lv-sweep: verification-attention throughput against the number of batched step tokens")
     ap.add_argument("--scale", type=float, default=1.0, help="shrink the number of problems (debugging only)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
@@ -193,6 +241,8 @@ def main():
     import torch
     from paper_2609_39334_b200 import synth
 
+    if args.workload == "lv-sweep":
+        return lv_sweep(args)
     cfg_idx = WORKLOADS[args.workload]
 
     # ---------------------------------------------------------------------------------------------- reference arm
