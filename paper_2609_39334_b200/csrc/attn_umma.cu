@@ -370,7 +370,10 @@ tile_items_umma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_
       // =================================================== MMA issuer ==========================================
       constexpr uint32_t idesc_qk = instr_desc_bf16(128, kKvTile, false);
       constexpr uint32_t idesc_pv = instr_desc_bf16(128, kHeadDim, true);
-      const uint32_t q_addr = smem_u32(smem + kOffQ);
+      // descriptors of the operand tiles at stage 0 / K-step 0; every MMA below derives its own with one add
+      const uint64_t q_desc0 = smem_desc_sw128(smem_u32(smem + kOffQ), 0, 1024);
+      const uint64_t k_desc0 = smem_desc_sw128(smem_u32(smem + kOffK), 0, 1024);
+      const uint64_t v_desc0 = smem_desc_sw128(smem_u32(smem + kOffV), 8192, 1024);
       bool ok = mbar_wait(&C.q_full, q_uses & 1, abort_flag);
       auto issue_qk = [&](int j) -> bool {
         const uint32_t gj = g_tile + j;
@@ -378,12 +381,13 @@ tile_items_umma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_
         // S[b] / P[b] of tile gj-2 is free: PV(gj-2) was issued earlier by this thread and MMAs execute in order
         if (!mbar_wait(&C.k_full[s], (gj / kStages) & 1, abort_flag)) return false;
         tc_fence_after();
-        const uint32_t k_addr = smem_u32(smem + kOffK + s * 16384);
+        const uint64_t k_desc = smem_desc_advance(k_desc0, static_cast<uint32_t>(s) * 16384u);
+        const uint32_t d_tmem = tmem + b * 64;
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {
-          const uint64_t ad = smem_desc_sw128(q_addr + (kk >> 2) * 16384 + (kk & 3) * 32, 0, 1024);
-          const uint64_t bd = smem_desc_sw128(k_addr + (kk >> 2) * 8192 + (kk & 3) * 32, 0, 1024);
-          mma_bf16_ss(tmem + b * 64, ad, bd, idesc_qk, kk > 0 ? 1u : 0u);
+          const uint64_t ad = smem_desc_advance(q_desc0, (kk >> 2) * 16384 + (kk & 3) * 32);
+          const uint64_t bd = smem_desc_advance(k_desc, (kk >> 2) * 8192 + (kk & 3) * 32);
+          mma_bf16_ss(d_tmem, ad, bd, idesc_qk, kk > 0 ? 1u : 0u);
         }
         mma_commit(&C.k_empty[s]);
         mma_commit(&C.s_full[b]);
@@ -399,12 +403,11 @@ tile_items_umma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_
              mbar_wait(&C.p_full[b], (gj >> 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t v_addr = smem_u32(smem + kOffV + s * 16384);
+        const uint64_t v_desc = smem_desc_advance(v_desc0, static_cast<uint32_t>(s) * 16384u);
+        const uint32_t o_tmem = tmem + kColO, p_tmem = tmem + b * 64;
 #pragma unroll
-        for (int kk = 0; kk < 4; ++kk) {
-          const uint64_t bd = smem_desc_sw128(v_addr + kk * 2048, 8192, 1024);
-          mma_bf16_ts(tmem + kColO, tmem + b * 64 + kk * 8, bd, idesc_pv, (j > 0 || kk > 0) ? 1u : 0u);
-        }
+        for (int kk = 0; kk < 4; ++kk)
+          mma_bf16_ts(o_tmem, p_tmem + kk * 8, smem_desc_advance(v_desc, kk * 2048), idesc_pv, (j > 0 || kk > 0) ? 1u : 0u);
         mma_commit(&C.v_empty[s]);
         mma_commit(&C.pv_done);
         if (j + 1 == n_tiles) mma_commit(&C.o_final);

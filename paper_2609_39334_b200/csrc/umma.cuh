@@ -149,6 +149,13 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr, uint32_t lbo
   d |= 2ull << 61;     // 128-byte swizzle
   return d;
 }
+// Descriptor of the same tile shifted by `bytes` (a multiple of 16 that keeps the start address below 256 KB): only
+// the low word changes, so the MMA-issuing thread spends one integer add per MMA instead of rebuilding the
+// descriptor (that thread's instruction stream is on the critical path: it can issue one MMA per ~56 clk at best).
+__device__ __forceinline__ uint64_t smem_desc_advance(uint64_t desc, uint32_t bytes) {
+  const uint32_t lo = static_cast<uint32_t>(desc) + (bytes >> 4);
+  return (desc & 0xffffffff00000000ull) | lo;
+}
 // Instruction descriptor: bf16 x bf16 -> fp32, dense, M x N tile, A K-major, B K-major or MN-major.
 __host__ __device__ constexpr uint32_t instr_desc_bf16(int m, int n, bool b_mn_major) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | (static_cast<uint32_t>(n >> 3) << 17) |
