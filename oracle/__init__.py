@@ -39,6 +39,7 @@ def _load():
             lib.ss_oracle_tree_attention.restype = ctypes.c_int32
             lib.ss_oracle_topk.restype = None
             lib.ss_oracle_early_prune.restype = None
+            lib.ss_oracle_branch_sample.restype = None
             _lib = lib
     return _lib
 
@@ -178,3 +179,21 @@ def early_prune(scores, verified, seg_offsets, k):
     lib.ss_oracle_early_prune(_p(sc), _p(ve), _p(seg_offsets), ctypes.c_int32(n_seg), ctypes.c_int32(k), _p(pruned),
                               _p(sel), _p(fin))
     return pruned[:n], sel[:n_seg, :k].reshape(n_seg, k), fin[:n_seg]
+
+
+def branch_sample(logits, draw_offsets, uniforms, temperature):
+    """logits f32 [n_seq][vocab], draw_offsets int64 [n_seq+1], uniforms f32 [total draws] ->
+    (tokens int32 [draws], seq int64 [draws], margin f64 [draws])."""
+    lib = _load()
+    logits = _c(logits, np.float32)
+    draw_offsets = _c(draw_offsets, np.int64)
+    uniforms = _c(uniforms, np.float32)
+    n_seq, vocab = int(logits.shape[0]), int(logits.shape[1])
+    n = int(draw_offsets[-1])
+    tokens = np.zeros(max(n, 1), np.int32)
+    seq = np.zeros(max(n, 1), np.int64)
+    margin = np.zeros(max(n, 1), np.float64)
+    un = uniforms if n else np.zeros(1, np.float32)
+    lib.ss_oracle_branch_sample(_p(logits), _p(draw_offsets), _p(un), ctypes.c_int32(n_seq), ctypes.c_int32(vocab),
+                                ctypes.c_double(float(temperature)), _p(tokens), _p(seq), _p(margin))
+    return tokens[:n], seq[:n], margin[:n]

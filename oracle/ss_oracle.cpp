@@ -16,6 +16,9 @@
 //   ss_oracle_early_prune     The same selection while only part of the candidates is verified: rule 1 (ranked
 //                             below the top-k of the verified ones => pruned) and rule 2 (k perfect scores =>
 //                             final), paper, Section "Early Pruning of Search Tree".
+//   ss_oracle_branch_sample   On-demand branching: the potential-many next-token draws of a sequence from one
+//                             logits row (paper, Section "Computation Deduplication"); inverse-CDF sampling with
+//                             the uniform random numbers passed in.
 //   ss_oracle_topk            Selection of the top-k candidates by score (paper, Section "Early Pruning of
 //                             Search Tree": a candidate ranked below the top-k cannot be selected;
 //                             top-k = N / M).  Plain stable sort.
@@ -287,6 +290,47 @@ void ss_oracle_early_prune(const float* scores, const uint8_t* verified, const i
       final_out[s] = 1;
       for (int32_t j = 0; j < k && j < static_cast<int32_t>(ver.size()); ++j)
         selected[static_cast<int64_t>(s) * k + j] = ver[j];
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// On-demand branching, sampling half (paper, Section "Computation Deduplication"): a sequence whose potential
+// size is n runs ONE forward pass and then draws n next tokens "as independent trials from the same
+// distribution"; equal draws are grouped afterwards (ss_oracle_dedup on (sequence, token) pairs gives the groups
+// and their cardinalities = the children's potential sizes).
+// Distribution: softmax(logits / temperature) over the vocabulary.  The random numbers are INPUTS: draw k of
+// sequence s uses uniforms[draw_offsets[s] + k] in [0, 1).  Inverse-CDF rule in fp64:
+//   e_v = exp((logit_v - max) / temperature),  C_v = e_0 + ... + e_v,  Z = C_{V-1},
+//   token = the smallest v with C_v > u * Z.
+// tokens_out[d] = sampled token of draw d, seq_out[d] = its sequence.  margin_out (may be null) receives, per
+// draw, min(|u*Z - C_{token-1}|, |C_token - u*Z|) / Z: how far the draw is from flipping to a neighbouring token.
+// ---------------------------------------------------------------------------------------------------------
+void ss_oracle_branch_sample(const float* logits, const int64_t* draw_offsets, const float* uniforms,
+                             int32_t n_seq, int32_t vocab, double temperature, int32_t* tokens_out,
+                             int64_t* seq_out, double* margin_out) {
+  std::vector<double> cdf(static_cast<size_t>(vocab > 0 ? vocab : 1));
+  for (int32_t s = 0; s < n_seq; ++s) {
+    const float* row = logits + static_cast<int64_t>(s) * vocab;
+    double mx = -std::numeric_limits<double>::infinity();
+    for (int32_t v = 0; v < vocab; ++v) mx = std::max(mx, static_cast<double>(row[v]));
+    double run = 0.0;
+    for (int32_t v = 0; v < vocab; ++v) {
+      run += std::exp((static_cast<double>(row[v]) - mx) / temperature);
+      cdf[v] = run;
+    }
+    const double Z = run;
+    for (int64_t d = draw_offsets[s]; d < draw_offsets[s + 1]; ++d) {
+      const double target = static_cast<double>(uniforms[d]) * Z;
+      int32_t tok = vocab - 1;
+      for (int32_t v = 0; v < vocab; ++v)
+        if (cdf[v] > target) { tok = v; break; }
+      tokens_out[d] = tok;
+      seq_out[d] = s;
+      if (margin_out) {
+        const double below = tok > 0 ? cdf[tok - 1] : 0.0;
+        margin_out[d] = std::min(std::fabs(target - below), std::fabs(cdf[tok] - target)) / Z;
+      }
     }
   }
 }

@@ -568,3 +568,64 @@ def test_early_prune_bruteforce_and_topk_consistency(seed):
     pruned, sel, fin = oracle.early_prune(sc2, ver, seg, k)
     surv, keep = oracle.topk(sc2, seg, k)
     assert np.array_equal(1 - pruned, keep) and np.array_equal(sel, surv) and fin.all()
+
+
+# =========================================================================================================
+# on-demand branching: sampling
+# =========================================================================================================
+def test_branch_sample_paper_worked_example():
+    kv = {}
+    for l in open(os.path.join(GOLDEN, "branch_sampling_example.txt")):
+        if l.strip() and not l.startswith("#"):
+            k, *v = l.split()
+            kv[k] = v
+    probs = np.asarray([float(x) for x in kv["probs"]])
+    with np.errstate(divide="ignore"):
+        logits = np.log(probs).astype(np.float32)[None, :]            # -inf where the probability is zero
+    u = np.asarray([float(x) for x in kv["uniforms"]], np.float32)
+    tokens, seq, _ = oracle.branch_sample(logits, [0, len(u)], u, float(kv["temperature"][0]))
+    assert list(tokens) == [int(x) for x in kv["tokens"]] and set(seq) == {0}
+    # grouping of the draws = dedup of (sequence, token) pairs; cardinalities = the children's potential sizes
+    r = oracle.dedup(tokens, np.arange(len(u) + 1), ctx_key=seq)
+    assert list(r["multiplicity"]) == [int(x) for x in kv["potentials"]]
+
+
+def test_branch_sample_closed_forms():
+    rng = np.random.default_rng(3)
+    V = 1000
+    u = rng.random(500).astype(np.float32)
+    # uniform logits: token = floor(u * V)
+    tokens, _, margin = oracle.branch_sample(np.zeros((1, V), np.float32), [0, 500], u, 0.7)
+    safe = margin > 1e-9
+    assert np.array_equal(tokens[safe], np.floor(u.astype(np.float64) * V).astype(np.int32)[safe])
+    # one token carries everything: always that token, whatever the temperature
+    lg = np.full((1, V), -np.inf, np.float32)
+    lg[0, 417] = 3.0
+    assert set(oracle.branch_sample(lg, [0, 500], u, 2.0)[0]) == {417}
+    # scaling logits and temperature together changes nothing; sorted uniforms give non-decreasing tokens
+    lg = rng.normal(size=(1, V)).astype(np.float32)
+    a = oracle.branch_sample(lg, [0, 500], u, 0.8)[0]
+    b = oracle.branch_sample(lg * 2, [0, 500], u, 1.6)[0]
+    assert np.array_equal(a, b)
+    us = np.sort(u)
+    assert np.all(np.diff(oracle.branch_sample(lg, [0, 500], us, 0.8)[0]) >= 0)
+
+
+def test_branch_sample_matches_numpy_inverse_cdf_and_frequencies():
+    rng = np.random.default_rng(4)
+    S, V, T = 5, 64, 0.8
+    lg = (rng.normal(size=(S, V)) * 2).astype(np.float32)
+    pot = rng.integers(0, 4000, size=S)
+    off = np.concatenate([[0], np.cumsum(pot)]).astype(np.int64)
+    u = rng.random(int(off[-1])).astype(np.float32)
+    tokens, seq, margin = oracle.branch_sample(lg, off, u, T)
+    for s in range(S):
+        p = np.exp((lg[s].astype(np.float64) - lg[s].max()) / T)
+        cdf = np.cumsum(p)
+        want = np.searchsorted(cdf, u[off[s]:off[s + 1]].astype(np.float64) * cdf[-1], side="right")
+        got = tokens[off[s]:off[s + 1]]
+        ok = margin[off[s]:off[s + 1]] > 1e-12
+        assert np.array_equal(got[ok], want[ok]) and np.all(seq[off[s]:off[s + 1]] == s)
+        if pot[s] > 2000:                                 # empirical frequencies follow the softmax
+            freq = np.bincount(got, minlength=V) / pot[s]
+            assert np.abs(freq - p / p.sum()).max() < 0.05
