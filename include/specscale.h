@@ -259,6 +259,31 @@ int32_t ss_early_prune(const float* scores, const uint8_t* verified, const int32
                        void* workspace, size_t workspace_bytes, void* stream);
 
 /* =========================================================================================================
+ * ss_branch_sample - the draws of on-demand branching.
+ *
+ * Paper: Section "Computation Deduplication" - a sequence with potential size n runs one forward pass and then
+ * samples n next tokens "as independent trials from the same distribution"; equal samples are grouped and every
+ * group becomes one child sequence whose potential size is the group's cardinality.  This call does the sampling;
+ * the grouping is ss_dedup_paths on the (sequence, token) pairs it returns (tok_ids = tokens_out with one token per
+ * path, ctx_key = seq_out): multiplicity_out are then the children's potential sizes.  (The paper batches the
+ * sampler by potential size because its sampler needs one output shape per call; one launch handles any mix here.)
+ *
+ * Distribution: softmax(logits / temperature).  The random numbers are inputs.  Rule (evaluated in fp64):
+ *   e_v = exp((logit_v - max) / temperature), C_v = e_0 + .. + e_v, token = the smallest v with C_v > u * C_{V-1}.
+ *
+ *   logits        fp32 [n_seq][vocab]   (-inf allowed: probability 0; at least one finite value per row)
+ *   draw_offsets  int64 [n_seq+1]       draws of sequence s are draw_offsets[s] .. draw_offsets[s+1]-1
+ *                                       (draw_offsets[s+1] - draw_offsets[s] = its potential size)
+ *   uniforms      fp32 [draw_offsets[n_seq]]  in [0, 1)
+ *   n_seq, vocab  host;  temperature host > 0
+ *   tokens_out    int32 [draws]   sampled token of every draw
+ *   seq_out       int64 [draws]   the sequence every draw belongs to
+ * Errors: SS_ERR_INVALID_ARG, SS_ERR_CUDA.
+ * ======================================================================================================= */
+int32_t ss_branch_sample(const float* logits, const int64_t* draw_offsets, const float* uniforms, int32_t n_seq,
+                         int32_t vocab, float temperature, int32_t* tokens_out, int64_t* seq_out, void* stream);
+
+/* =========================================================================================================
  * Diagnostics
  * ======================================================================================================= */
 /* Number of kernels this library has launched in this process since it was loaded (host counter). */

@@ -34,6 +34,7 @@ EXPORTS = [
     "ss_tree_attention_workspace_bytes", "ss_tree_attention", "ss_topk_workspace_bytes", "ss_topk_prune",
     "ss_launch_count", "ss_debug_umma_tile", "ss_profile_enable", "ss_profile_read",
     "ss_dedup_paths_static", "ss_debug_tile_kernel_occupancy", "ss_early_prune",
+    "ss_branch_sample",
 ]
 PHASES = ["plan", "tiles", "leaves", "generic", "merge"]
 
@@ -238,6 +239,16 @@ def ss_early_prune(scores, verified, seg_offsets, n_segments, n_total, k, pruned
                               ctypes.c_size_t(workspace.numel() if workspace is not None else 0), _stream(stream))
     if check:
         _check(rc, "ss_early_prune")
+    return rc
+
+
+def ss_branch_sample(logits, draw_offsets, uniforms, n_seq, vocab, temperature, tokens_out, seq_out, stream=None,
+                     check=True) -> int:
+    rc = lib().ss_branch_sample(_ptr(logits), _ptr(draw_offsets), _ptr(uniforms), ctypes.c_int32(n_seq),
+                                ctypes.c_int32(vocab), ctypes.c_float(temperature), _ptr(tokens_out), _ptr(seq_out),
+                                _stream(stream))
+    if check:
+        _check(rc, "ss_branch_sample")
     return rc
 
 
