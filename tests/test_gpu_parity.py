@@ -467,3 +467,41 @@ def test_attention_reports_too_small_workspace_from_the_device():
     # host-side check: a workspace smaller than the query result is refused before any launch
     rc = B.ss_tree_attention(pipe.desc, ws[:1024], check=False)
     assert rc == B.SS_ERR_WORKSPACE_TOO_SMALL
+
+
+# =========================================================================================================
+# sizes at the edges of the supported range
+# =========================================================================================================
+EDGE_SHAPES = [
+    # one very long path (decode and verification): many key tiles, one item per kv head
+    ("long_decode", 8, 2, [16384], [1], 1, (2000, 2100), lambda i, n, rng: 1),
+    ("long_verify", 8, 2, [8192], [2], 1, (100, 900), lambda i, n, rng: 128),
+    # GQA group of 1 (128 tokens per tile) and of 128 (one token per tile), maximum step length
+    ("gqa1_verify", 2, 2, [64], [3], 1, (0, 200), lambda i, n, rng: 128),
+    ("gqa128_verify", 128, 1, [64], [2], 1, (0, 100), lambda i, n, rng: 5),
+    # many tiny problems (more nodes than SMs), leaves that end exactly on page / tile boundaries
+    ("many_problems", 12, 2, [32], [2], 300, (0, 20), lambda i, n, rng: 1 + (i % 2) * 15),
+    ("exact_boundaries", 8, 2, [64], [4], 2, (64, 64), lambda i, n, rng: 1 + (i % 2) * 63),
+    # depth at the limit: 15 shared levels + leaf
+    ("depth16", 4, 2, [16] * 15, [1] * 14 + [3], 1, (1, 40), lambda i, n, rng: 1 + (i % 2) * 8),
+]
+
+
+@pytest.mark.parametrize("shape", EDGE_SHAPES, ids=[s[0] for s in EDGE_SHAPES])
+def test_attention_edge_sizes(shape):
+    name, Hq, Hkv, levels, fanout, problems, leaf, qfn = shape
+    w = synth.build_tree_workload(name, 4321, Hq, Hkv, levels, fanout, problems, leaf, qfn)
+    r, ref = attention_only(w)
+    check_attention(r, w, ref, max_paths=24)
+
+
+def test_dedup_large_batch():
+    """One million candidate paths (far beyond the benchmark sizes): still bit-exact."""
+    rng = np.random.default_rng(2024)
+    n = 1_000_000
+    ids, off, ctx, slot = dedup_case(rng, n, 30, 3, 8)
+    got = run_dedup(ids, off, ctx, slot)
+    want = oracle.dedup(ids, off, ctx, slot)
+    assert got["num_unique"] == want["num_unique"]
+    for key in ("canon", "path_to_unique", "unique_paths", "multiplicity", "slot_out"):
+        assert np.array_equal(got[key], want[key]), key
