@@ -11,6 +11,8 @@
 //   4. compact   exclusive scan of (canon[i] == i) in index order -> ranks; unique list, multiplicities
 //                (integer atomics: order-independent), path_to_unique, slot remap
 // Hash collisions only cost time: equality is always decided on the token ids themselves.
+// Batches of up to 4096 paths run the same four steps in two launches (the last block to finish a grid-parallel
+// step runs the single-block step that follows it; the sort is a bitonic network in shared memory).
 #include "common.cuh"
 
 namespace ss {
@@ -28,13 +30,10 @@ __device__ __forceinline__ uint64_t mix64(uint64_t x) {   // splitmix64 finalise
   return x;
 }
 
-__global__ void hash_kernel(const int32_t* __restrict__ tok_ids, const int64_t* __restrict__ tok_offsets,
-                            const int64_t* __restrict__ ctx_key, int n, uint32_t weak, uint64_t* __restrict__ hash64,
-                            uint32_t* __restrict__ keys, uint32_t* __restrict__ idx) {
-  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  const int lane = threadIdx.x & 31;
-  if (warp >= n) return;
-  const int64_t lo = tok_offsets[warp], hi = tok_offsets[warp + 1];
+// Whole warp: 64-bit hash of path `path` (returned to every lane).
+__device__ __forceinline__ uint64_t hash_path(const int32_t* __restrict__ tok_ids, const int64_t* __restrict__ tok_offsets,
+                                              const int64_t* __restrict__ ctx_key, int path, uint32_t weak, int lane) {
+  const int64_t lo = tok_offsets[path], hi = tok_offsets[path + 1];
   uint64_t acc = 0;
   for (int64_t j = lo + lane; j < hi; j += 32) {
     const uint64_t t = static_cast<uint32_t>(tok_ids[j]);
@@ -42,12 +41,26 @@ __global__ void hash_kernel(const int32_t* __restrict__ tok_ids, const int64_t* 
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  uint64_t h = mix64(acc ^ mix64(static_cast<uint64_t>(hi - lo) + 0x632be59bd9b4e019ull));
+  if (ctx_key) h = mix64(h ^ mix64(static_cast<uint64_t>(ctx_key[path]) + 0x2545f4914f6cdd1dull));
+  if (weak) h &= 0xffull;                       // SS_FLAG_WEAK_HASH: force collisions
+  return h;
+}
+
+__device__ __forceinline__ uint32_t sort_key_of(uint64_t h, uint32_t weak) {
+  return weak ? static_cast<uint32_t>(h) : static_cast<uint32_t>(h >> 32);
+}
+
+__global__ void hash_kernel(const int32_t* __restrict__ tok_ids, const int64_t* __restrict__ tok_offsets,
+                            const int64_t* __restrict__ ctx_key, int n, uint32_t weak, uint64_t* __restrict__ hash64,
+                            uint32_t* __restrict__ keys, uint32_t* __restrict__ idx) {
+  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (warp >= n) return;
+  const uint64_t h = hash_path(tok_ids, tok_offsets, ctx_key, warp, weak, lane);
   if (lane == 0) {
-    uint64_t h = mix64(acc ^ mix64(static_cast<uint64_t>(hi - lo) + 0x632be59bd9b4e019ull));
-    if (ctx_key) h = mix64(h ^ mix64(static_cast<uint64_t>(ctx_key[warp]) + 0x2545f4914f6cdd1dull));
-    if (weak) h &= 0xffull;                     // SS_FLAG_WEAK_HASH: force collisions
     hash64[warp] = h;
-    keys[warp] = weak ? static_cast<uint32_t>(h) : static_cast<uint32_t>(h >> 32);
+    keys[warp] = sort_key_of(h, weak);
     idx[warp] = warp;
   }
 }
@@ -142,13 +155,14 @@ __global__ void rs_scatter(const uint32_t* __restrict__ keys_in, const uint32_t*
 }
 
 // ---- exact matching inside equal-key runs ---------------------------------------------------------------
-__global__ void match_kernel(const uint32_t* __restrict__ keys, const uint32_t* __restrict__ idx, int n,
-                             const uint64_t* __restrict__ hash64, const int32_t* __restrict__ tok_ids,
-                             const int64_t* __restrict__ tok_offsets, const int64_t* __restrict__ ctx_key,
-                             int32_t* __restrict__ canon_out) {
-  const int s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  const int lane = threadIdx.x & 31;
-  if (s >= n) return;
+// Whole warp: canonical representative of the path at sorted position s.
+// (keys, idx, hash64 carry no __restrict__ here: the single-block kernel writes them before it reads them.)
+__device__ __forceinline__ void match_sorted_position(const uint32_t* keys, const uint32_t* idx, int s,
+                                                      const uint64_t* hash64,
+                                                      const int32_t* __restrict__ tok_ids,
+                                                      const int64_t* __restrict__ tok_offsets,
+                                                      const int64_t* __restrict__ ctx_key,
+                                                      int32_t* canon_out, int lane) {
   const uint32_t key = keys[s];
   const int i = static_cast<int>(idx[s]);
   // start of the run of equal keys (lower bound)
@@ -187,10 +201,19 @@ __global__ void match_kernel(const uint32_t* __restrict__ keys, const uint32_t* 
   if (lane == 0) canon_out[i] = canon;
 }
 
+__global__ void match_kernel(const uint32_t* __restrict__ keys, const uint32_t* __restrict__ idx, int n,
+                             const uint64_t* __restrict__ hash64, const int32_t* __restrict__ tok_ids,
+                             const int64_t* __restrict__ tok_offsets, const int64_t* __restrict__ ctx_key,
+                             int32_t* __restrict__ canon_out) {
+  const int s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  if (s >= n) return;
+  match_sorted_position(keys, idx, s, hash64, tok_ids, tok_offsets, ctx_key, canon_out, threadIdx.x & 31);
+}
+
 // ---- compaction ----------------------------------------------------------------------------------------------
 // One block: rank[i] = number of unique paths with a smaller index; also clears the multiplicities.
-__global__ void rank_kernel(const int32_t* __restrict__ canon, int n, int32_t* __restrict__ rank,
-                            int32_t* __restrict__ multiplicity, int32_t* __restrict__ num_unique) {
+__device__ __forceinline__ void rank_block(const int32_t* canon, int n, int32_t* rank, int32_t* multiplicity,
+                                           int32_t* num_unique) {
   __shared__ int warp_tot[32];
   __shared__ int carry_s;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
@@ -223,18 +246,100 @@ __global__ void rank_kernel(const int32_t* __restrict__ canon, int n, int32_t* _
   if (threadIdx.x == 0) *num_unique = carry_s;
 }
 
-__global__ void finalize_kernel(const int32_t* __restrict__ canon, const int32_t* __restrict__ rank, int n,
-                                const int32_t* __restrict__ slot_in, int32_t* __restrict__ path_to_unique,
-                                int32_t* __restrict__ unique_paths, int32_t* __restrict__ multiplicity,
-                                int32_t* __restrict__ slot_out) {
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= n) return;
+__global__ void rank_kernel(const int32_t* __restrict__ canon, int n, int32_t* __restrict__ rank,
+                            int32_t* __restrict__ multiplicity, int32_t* __restrict__ num_unique) {
+  rank_block(canon, n, rank, multiplicity, num_unique);
+}
+
+__device__ __forceinline__ void finalize_path(const int32_t* canon, const int32_t* rank, int i,
+                                              const int32_t* __restrict__ slot_in, int32_t* path_to_unique,
+                                              int32_t* unique_paths, int32_t* multiplicity, int32_t* slot_out) {
   const int c = canon[i];
   const int r = rank[c];
   path_to_unique[i] = r;
   if (c == i) unique_paths[r] = i;
   atomicAdd(&multiplicity[r], 1);
   if (slot_out) slot_out[i] = slot_in[c];
+}
+
+__global__ void finalize_kernel(const int32_t* __restrict__ canon, const int32_t* __restrict__ rank, int n,
+                                const int32_t* __restrict__ slot_in, int32_t* __restrict__ path_to_unique,
+                                int32_t* __restrict__ unique_paths, int32_t* __restrict__ multiplicity,
+                                int32_t* __restrict__ slot_out) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  finalize_path(canon, rank, i, slot_in, path_to_unique, unique_paths, multiplicity, slot_out);
+}
+
+// ---- small batches ---------------------------------------------------------------------------------------------
+// A batch of a few thousand paths is launch-latency bound: the multi-launch path above is ~17 dependent launches.
+// Here the same four steps take two: the grid-parallel steps (hash, match) stay grid-parallel, and the block that
+// finishes LAST (a counter in the workspace, zeroed by a memset ahead of the first kernel) runs the single-block step
+// that follows (bitonic sort in shared memory; rank scan + finalize).
+constexpr int kSmallMax = 4096;
+constexpr int kSmallThreads = 1024;
+constexpr int kSmallWarps = kSmallThreads / 32;
+
+// True in every thread of the block that arrives last; its reads come after all other blocks' writes.
+__device__ __forceinline__ bool last_block_arrives(unsigned int* counter) {
+  __shared__ bool s_last;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) s_last = atomicAdd(counter, 1u) == gridDim.x - 1;
+  __syncthreads();
+  if (s_last) __threadfence();
+  return s_last;
+}
+
+__global__ void __launch_bounds__(kSmallThreads)
+small_hash_sort_kernel(const int32_t* __restrict__ tok_ids, const int64_t* __restrict__ tok_offsets,
+                       const int64_t* __restrict__ ctx_key, int n, uint32_t weak, uint64_t* hash64, uint32_t* keys,
+                       uint32_t* idx, unsigned int* counter) {
+  __shared__ uint64_t skey[kSmallMax];            // (sort key << 32 | path index): distinct, so the order is total
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int p = blockIdx.x * kSmallWarps + (tid >> 5);
+  if (p < n) {
+    const uint64_t h = hash_path(tok_ids, tok_offsets, ctx_key, p, weak, lane);
+    if (lane == 0) hash64[p] = h;
+  }
+  if (!last_block_arrives(counter)) return;
+  int n_pad = 1;
+  while (n_pad < n) n_pad <<= 1;
+  for (int i = tid; i < n_pad; i += blockDim.x)
+    skey[i] = i < n ? (static_cast<uint64_t>(sort_key_of(__ldcg(hash64 + i), weak)) << 32) | static_cast<uint32_t>(i)
+                    : ~0ull;
+  __syncthreads();
+  for (int size = 2; size <= n_pad; size <<= 1)
+    for (int stride = size >> 1; stride > 0; stride >>= 1) {
+      for (int t = tid; t < (n_pad >> 1); t += blockDim.x) {
+        const int lo = ((t / stride) * (stride << 1)) + (t % stride);
+        const int hi = lo + stride;
+        const bool up = ((lo & size) == 0);
+        const uint64_t a = skey[lo], b = skey[hi];
+        if ((a > b) == up) { skey[lo] = b; skey[hi] = a; }
+      }
+      __syncthreads();
+    }
+  for (int i = tid; i < n; i += blockDim.x) {
+    keys[i] = static_cast<uint32_t>(skey[i] >> 32);
+    idx[i] = static_cast<uint32_t>(skey[i]);
+  }
+}
+
+__global__ void __launch_bounds__(kSmallThreads)
+small_match_finalize_kernel(const uint32_t* __restrict__ keys, const uint32_t* __restrict__ idx, int n,
+                            const uint64_t* __restrict__ hash64, const int32_t* __restrict__ tok_ids,
+                            const int64_t* __restrict__ tok_offsets, const int64_t* __restrict__ ctx_key,
+                            const int32_t* __restrict__ slot_in, int32_t* canon_out, int32_t* rank,
+                            int32_t* path_to_unique, int32_t* unique_paths, int32_t* multiplicity, int32_t* slot_out,
+                            int32_t* num_unique, unsigned int* counter) {
+  const int s = blockIdx.x * kSmallWarps + (threadIdx.x >> 5);
+  if (s < n) match_sorted_position(keys, idx, s, hash64, tok_ids, tok_offsets, ctx_key, canon_out, threadIdx.x & 31);
+  if (!last_block_arrives(counter)) return;
+  rank_block(canon_out, n, rank, multiplicity, num_unique);     // canon_out was not read before: no stale L1 lines
+  __syncthreads();
+  for (int i = threadIdx.x; i < n; i += blockDim.x)
+    finalize_path(canon_out, rank, i, slot_in, path_to_unique, unique_paths, multiplicity, slot_out);
 }
 
 __global__ void zero_scalar_kernel(int32_t* p) { *p = 0; }
@@ -301,6 +406,20 @@ extern "C" int32_t ss_dedup_paths(const int32_t* tok_ids, const int64_t* tok_off
 
   const int n = n_paths;
   const uint32_t weak = (flags & SS_FLAG_WEAK_HASH) ? 1u : 0u;
+  if (n <= kSmallMax) {
+    unsigned int* counters = reinterpret_cast<unsigned int*>(hist);      // the sort histogram is unused on this path
+    if (cudaMemsetAsync(counters, 0, 2 * sizeof(unsigned int), st) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return SS_ERR_CUDA;
+    }
+    const int blocks = (n + kSmallWarps - 1) / kSmallWarps;
+    SS_LAUNCH(small_hash_sort_kernel, blocks, kSmallThreads, 0, st, tok_ids, tok_offsets, ctx_key, n, weak, hash64, keys_a,
+              idx_a, counters);
+    SS_LAUNCH(small_match_finalize_kernel, blocks, kSmallThreads, 0, st, keys_a, idx_a, n, hash64, tok_ids, tok_offsets,
+              ctx_key, slot_in, canon_out, rank, path_to_unique_out, unique_paths_out, multiplicity_out, slot_out,
+              num_unique_out, counters + 1);
+    return SS_OK;
+  }
   const int warps_per_block = 8;
   const int warp_blocks = (n + warps_per_block - 1) / warps_per_block;
   SS_LAUNCH(hash_kernel, warp_blocks, warps_per_block * 32, 0, st, tok_ids, tok_offsets, ctx_key, n, weak, hash64,

@@ -153,7 +153,7 @@ def dedup_case(rng, n, alphabet, max_len, n_ctx):
 
 @pytest.mark.parametrize("flags", [0, B.SS_FLAG_WEAK_HASH])
 @pytest.mark.parametrize("n,alphabet,max_len,n_ctx", [
-    (1, 3, 4, 1), (2, 2, 2, 1), (37, 2, 3, 2), (300, 3, 5, 2), (2049, 4, 6, 3), (5000, 2, 40, 1), (20000, 50, 3, 4),
+    (1, 3, 4, 1), (2, 2, 2, 1), (37, 2, 3, 2), (300, 3, 5, 2), (2049, 4, 6, 3), (4096, 3, 5, 2), (4097, 3, 5, 2), (5000, 2, 40, 1), (20000, 50, 3, 4),
 ])
 def test_dedup_random_collision_heavy(n, alphabet, max_len, n_ctx, flags):
     rng = np.random.default_rng(n * 31 + alphabet)
