@@ -97,6 +97,28 @@ int32_t ss_dedup_paths(const int32_t* tok_ids, const int64_t* tok_offsets, const
                        int32_t* slot_out, int32_t* num_unique_out, void* workspace, size_t workspace_bytes,
                        void* stream);
 
+/* ss_gather_unique_paths - descriptor rows of the unique paths, in the layout ss_tree_attention takes.
+ *
+ * (Paper, Section "Computation Deduplication": a group of equal candidates gets ONE forward pass; this builds
+ * the per-path arguments of that pass from the grouping.)  For p < U = *num_unique, with s = unique_paths[p]:
+ *   u_leaf_out[p] = path_leaf_node[s],  u_q_len_out[p] = path_q_len[s],  u_q_src_out[p] = q_offsets[s]
+ *   u_q_offsets_out[p+1] = u_q_len_out[0] + ... + u_q_len_out[p]          (u_q_offsets_out[0] = 0)
+ * and for U <= p < n_paths: u_leaf_out[p] = -1, u_q_len_out[p] = 0, u_q_src_out[p] = 0,
+ * u_q_offsets_out[p+1] = u_q_offsets_out[U].  Query rows are not moved: pass u_q_src_out as q_src_offsets.
+ *
+ *   unique_paths    int32 [n_paths]    device; first U entries used (ss_dedup_paths' unique_paths_out)
+ *   num_unique      int32 [1]          device; U, clamped to [0, n_paths]
+ *   n_paths         host, >= 0
+ *   path_leaf_node  int32 [n_paths]    device; per LOGICAL path
+ *   path_q_len      int32 [n_paths]    device
+ *   q_offsets       int64 [n_paths+1]  device; row of each logical path's first query token
+ *   u_leaf_out, u_q_len_out  int32 [n_paths];  u_q_offsets_out  int64 [n_paths+1];  u_q_src_out  int64 [n_paths]
+ * No workspace, no host synchronisation; one launch on `stream`.  Errors: SS_ERR_INVALID_ARG, SS_ERR_CUDA. */
+int32_t ss_gather_unique_paths(const int32_t* unique_paths, const int32_t* num_unique, int32_t n_paths,
+                               const int32_t* path_leaf_node, const int32_t* path_q_len, const int64_t* q_offsets,
+                               int32_t* u_leaf_out, int32_t* u_q_len_out, int64_t* u_q_offsets_out,
+                               int64_t* u_q_src_out, void* stream);
+
 /* ss_dedup_paths_static - ss_dedup_paths without a caller workspace and without any allocation.
  *
  * (The paper has no counterpart; this is a convenience of the library.)  It exists for callers that cannot ask
@@ -282,6 +304,73 @@ int32_t ss_early_prune(const float* scores, const uint8_t* verified, const int32
  * ======================================================================================================= */
 int32_t ss_branch_sample(const float* logits, const int64_t* draw_offsets, const float* uniforms, int32_t n_seq,
                          int32_t vocab, float temperature, int32_t* tokens_out, int64_t* seq_out, void* stream);
+
+/* =========================================================================================================
+ * ss_candidate_step_host - one pass of the whole path for per-step data that lives in HOST memory.
+ *
+ * Paper: the system overview figure and Sections "Computation Deduplication", "Lazy Verification" and "Early
+ * Pruning of Search Tree" - per expansion / verification step the candidates are deduplicated, the unique ones get one attention pass over the
+ * shared KV prefixes, and the scored candidates are pruned to the top-k.  This call is that sequence for a caller
+ * whose candidates, query activations and scores are produced on the host side of the bus:
+ *   asynchronous copies host -> device of every per-step input  ->  ss_dedup_paths  ->  ss_gather_unique_paths  ->
+ *   ss_tree_attention (queries read in place through the gathered offsets)  ->  ss_topk_prune  ->
+ *   asynchronous copies device -> host of every result.
+ * Everything is enqueued on `stream`; the call does not synchronise, and it allocates nothing: staging buffers,
+ * results and the workspaces of the three calls are carved out of `device_arena` (caller-owned, 256-byte aligned,
+ * >= ss_candidate_step_host_arena_bytes).  The KV pool and the tree stay resident on the device: they are the
+ * cache state of the method, described by the resident fields of `attn` (flags, heads, sm_scale, pool, strides,
+ * tree arrays, total_node_pages, max_depth, max_decode_paths); the path, query and output fields of `attn` are
+ * ignored.  Host buffers should be page-locked, else the copies are synchronous (results are the same).  A caller
+ * that alternates between two or three (arena, stream, host buffer) sets overlaps the copies of one step with the
+ * kernels of another.  Results are valid once `stream` has drained; *device_status then holds what
+ * ss_last_device_status would report for the attention call.
+ *
+ * Inputs (host): as the arguments of the same name of ss_dedup_paths, ss_gather_unique_paths, ss_tree_attention
+ * (q: bf16 [total_q][Hq][128] in logical-candidate order) and ss_topk_prune.  ctx_key may be NULL; slot_in and
+ * slot_out must both be given or both be NULL; lse may be NULL.
+ * Results (host): canon, path_to_unique, unique_paths, multiplicity, slot_out [n_paths], num_unique [1],
+ * u_q_offsets int64 [n_paths+1] (rows of out / lse of unique path p: u_q_offsets[p] .. u_q_offsets[p+1]-1),
+ * out bf16 [total_q][Hq][128], lse fp32 [total_q][Hq], survivors int32 [n_segments][top_k], keep uint8 [n_paths],
+ * device_status int32 [1].
+ * Errors: SS_ERR_INVALID_ARG, SS_ERR_WORKSPACE_TOO_SMALL, SS_ERR_UNSUPPORTED, SS_ERR_CUDA (host); the device-side
+ * errors of ss_tree_attention arrive in *device_status.
+ * ======================================================================================================= */
+typedef struct ss_host_step {
+  uint32_t struct_size;              /* = sizeof(ss_host_step_t) */
+  uint32_t dedup_flags;              /* 0 or SS_FLAG_WEAK_HASH */
+  const ss_attn_desc_t* attn;        /* host; resident fields only (see above) */
+  int32_t n_paths, n_segments, top_k, reserved0;
+  int64_t total_tok;                 /* = tok_offsets[n_paths] - tok_offsets[0], and tok_offsets[0] must be 0 */
+  int64_t total_q;                   /* = q_offsets[n_paths], and q_offsets[0] must be 0 */
+  /* per-step inputs, host memory */
+  const int32_t* tok_ids;
+  const int64_t* tok_offsets;
+  const int64_t* ctx_key;
+  const int32_t* slot_in;
+  const int32_t* path_leaf_node;
+  const int32_t* path_q_len;
+  const int64_t* q_offsets;
+  const void* q;
+  const float* scores;
+  const int32_t* seg_offsets;
+  /* results, host memory */
+  int32_t* canon;
+  int32_t* path_to_unique;
+  int32_t* unique_paths;
+  int32_t* multiplicity;
+  int32_t* slot_out;
+  int32_t* num_unique;
+  int64_t* u_q_offsets;
+  void* out;
+  float* lse;
+  int32_t* survivors;
+  uint8_t* keep;
+  int32_t* device_status;
+} ss_host_step_t;
+
+int32_t ss_candidate_step_host_arena_bytes(const ss_host_step_t* step /* host */, size_t* out_bytes /* host */);
+int32_t ss_candidate_step_host(const ss_host_step_t* step /* host */, void* device_arena, size_t arena_bytes,
+                               void* stream);
 
 /* =========================================================================================================
  * Diagnostics

@@ -197,3 +197,22 @@ def branch_sample(logits, draw_offsets, uniforms, temperature):
     lib.ss_oracle_branch_sample(_p(logits), _p(draw_offsets), _p(un), ctypes.c_int32(n_seq), ctypes.c_int32(vocab),
                                 ctypes.c_double(float(temperature)), _p(tokens), _p(seq), _p(margin))
     return tokens[:n], seq[:n], margin[:n]
+
+
+def gather_unique(unique_paths, num_unique, n_paths, path_leaf_node, path_q_len, q_offsets):
+    """Per-path arguments of the single forward pass a group of equal candidates gets (paper, Section
+    "Computation Deduplication"): the descriptor rows of the group representatives, in order, written as plain
+    loops.  Entries past the number of unique paths are inert (-1 / 0 / 0, offsets stay at the total)."""
+    U = max(0, min(int(num_unique), int(n_paths)))
+    u_leaf = np.full(n_paths, -1, np.int32)
+    u_q_len = np.zeros(n_paths, np.int32)
+    u_q_src = np.zeros(n_paths, np.int64)
+    u_q_offsets = np.zeros(n_paths + 1, np.int64)
+    for p in range(n_paths):
+        if p < U:
+            s = int(unique_paths[p])
+            u_leaf[p] = path_leaf_node[s]
+            u_q_len[p] = path_q_len[s]
+            u_q_src[p] = q_offsets[s]
+        u_q_offsets[p + 1] = u_q_offsets[p] + int(u_q_len[p])
+    return dict(u_leaf=u_leaf, u_q_len=u_q_len, u_q_offsets=u_q_offsets, u_q_src=u_q_src)

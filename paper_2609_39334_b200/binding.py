@@ -34,7 +34,7 @@ EXPORTS = [
     "ss_tree_attention_workspace_bytes", "ss_tree_attention", "ss_topk_workspace_bytes", "ss_topk_prune",
     "ss_launch_count", "ss_debug_umma_tile", "ss_profile_enable", "ss_profile_read",
     "ss_dedup_paths_static", "ss_debug_tile_kernel_occupancy", "ss_early_prune",
-    "ss_branch_sample",
+    "ss_branch_sample", "ss_gather_unique_paths", "ss_candidate_step_host_arena_bytes", "ss_candidate_step_host",
 ]
 PHASES = ["plan", "tiles", "leaves", "generic", "merge"]
 
@@ -155,6 +155,77 @@ def ss_dedup_paths_static(tok_ids, tok_offsets, ctx_key, slot_in, n_paths, flags
                                      _ptr(slot_out), _ptr(num_unique_out), _stream(stream))
     if check:
         _check(rc, "ss_dedup_paths_static")
+    return rc
+
+
+def ss_gather_unique_paths(unique_paths, num_unique, n_paths, path_leaf_node, path_q_len, q_offsets, u_leaf_out,
+                           u_q_len_out, u_q_offsets_out, u_q_src_out, stream=None, check=True) -> int:
+    """Descriptor rows of the unique paths (leaf node, query length, query offsets, source query row) gathered by
+    `unique_paths`, ready to be passed to ss_tree_attention."""
+    rc = lib().ss_gather_unique_paths(_ptr(unique_paths), _ptr(num_unique), ctypes.c_int32(n_paths),
+                                      _ptr(path_leaf_node), _ptr(path_q_len), _ptr(q_offsets), _ptr(u_leaf_out),
+                                      _ptr(u_q_len_out), _ptr(u_q_offsets_out), _ptr(u_q_src_out), _stream(stream))
+    if check:
+        _check(rc, "ss_gather_unique_paths")
+    return rc
+
+
+class ss_host_step_t(ctypes.Structure):
+    _fields_ = [
+        ("struct_size", ctypes.c_uint32), ("dedup_flags", ctypes.c_uint32),
+        ("attn", ctypes.c_void_p),
+        ("n_paths", ctypes.c_int32), ("n_segments", ctypes.c_int32), ("top_k", ctypes.c_int32),
+        ("reserved0", ctypes.c_int32),
+        ("total_tok", ctypes.c_int64), ("total_q", ctypes.c_int64),
+    ] + [(n, ctypes.c_void_p) for n in (
+        "tok_ids", "tok_offsets", "ctx_key", "slot_in", "path_leaf_node", "path_q_len", "q_offsets", "q", "scores",
+        "seg_offsets", "canon", "path_to_unique", "unique_paths", "multiplicity", "slot_out", "num_unique",
+        "u_q_offsets", "out", "lse", "survivors", "keep", "device_status")]
+
+
+HOST_STEP_INPUTS = ("tok_ids", "tok_offsets", "ctx_key", "slot_in", "path_leaf_node", "path_q_len", "q_offsets", "q",
+                    "scores", "seg_offsets")
+HOST_STEP_RESULTS = ("canon", "path_to_unique", "unique_paths", "multiplicity", "slot_out", "num_unique",
+                     "u_q_offsets", "out", "lse", "survivors", "keep", "device_status")
+
+
+def make_host_step(attn_desc: "ss_attn_desc_t", *, n_paths, n_segments, top_k, total_tok, total_q, host_in: dict,
+                   host_out: dict, dedup_flags=0) -> ss_host_step_t:
+    """Fills ss_host_step_t from dictionaries of HOST tensors (page-locked for asynchronous copies) keyed by the field
+    names.  The returned object keeps references to the descriptor and the tensors."""
+    s = ss_host_step_t()
+    s.struct_size = ctypes.sizeof(ss_host_step_t)
+    s.dedup_flags = dedup_flags
+    s.attn = ctypes.addressof(attn_desc)
+    s.n_paths, s.n_segments, s.top_k = int(n_paths), int(n_segments), int(top_k)
+    s.total_tok, s.total_q = int(total_tok), int(total_q)
+    for name in HOST_STEP_INPUTS:
+        t = host_in.get(name)
+        assert t is None or (not t.is_cuda and t.is_contiguous()), name
+        setattr(s, name, t.data_ptr() if t is not None and t.numel() else None)
+    for name in HOST_STEP_RESULTS:
+        t = host_out.get(name)
+        assert t is None or (not t.is_cuda and t.is_contiguous()), name
+        setattr(s, name, t.data_ptr() if t is not None and t.numel() else None)
+    s._keep = (attn_desc, host_in, host_out)
+    return s
+
+
+def ss_candidate_step_host_arena_bytes(step: ss_host_step_t) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().ss_candidate_step_host_arena_bytes(ctypes.byref(step), ctypes.byref(out)),
+           "ss_candidate_step_host_arena_bytes")
+    return int(out.value)
+
+
+def ss_candidate_step_host(step: ss_host_step_t, device_arena: torch.Tensor, stream=None, check=True) -> int:
+    """The whole path for host-resident per-step data: copies in, dedup, gather, attention, top-k, copies out; all
+    asynchronous on `stream`."""
+    rc = lib().ss_candidate_step_host(ctypes.byref(step), _ptr(device_arena),
+                                      ctypes.c_size_t(device_arena.numel() * device_arena.element_size()),
+                                      _stream(stream))
+    if check:
+        _check(rc, "ss_candidate_step_host")
     return rc
 
 

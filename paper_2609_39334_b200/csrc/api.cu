@@ -1,8 +1,15 @@
 // Status strings, device-status read-back and the launch counter.
+#include <cstdlib>
+
 #include "common.cuh"
 
 namespace ss {
 long long g_launch_count = 0;
+
+bool pdl_enabled() {
+  static const bool on = std::getenv("SS_NO_PDL") == nullptr;
+  return on;
+}
 }
 
 extern "C" const char* ss_status_string(int32_t status) {

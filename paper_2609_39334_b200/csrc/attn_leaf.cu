@@ -39,6 +39,7 @@ constexpr int kLeafWarps = 4;
 // TWO: the GQA group has more than 8 rows (rows gid and gid+8 of the MMA tile are both live).
 template <bool TWO>
 __global__ void __launch_bounds__(kLeafWarps * 32) leaf_items_kernel(const Params P) {
+  ss::grid_dependency_enter();
   if (P.hdr->status != SS_OK) return;
   const int lane = threadIdx.x & 31;
   const int gid = lane >> 2, tig = lane & 3;

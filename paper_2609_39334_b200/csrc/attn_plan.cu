@@ -77,6 +77,7 @@ __device__ __forceinline__ int live_paths(const Params& P) {
 
 // ---- nodes: depth and number of keys before the node -------------------------------------------------------------
 __global__ void __launch_bounds__(kGridThreads) plan_nodes_kernel(const Params P) {
+  ss::grid_dependency_enter();
   PlanHeader* hdr = P.hdr;
   const int64_t gtid = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   const int64_t gsize = static_cast<int64_t>(gridDim.x) * blockDim.x;
@@ -116,6 +117,7 @@ __global__ void __launch_bounds__(kGridThreads) plan_nodes_kernel(const Params P
 
 // ---- paths: class, kv length, membership counts of every chain node ------------------------------------------------
 __global__ void __launch_bounds__(kGridThreads) plan_paths_kernel(const Params P) {
+  ss::grid_dependency_enter();
   PlanHeader* hdr = P.hdr;
   if (hdr->status != SS_OK) return;          // no barrier in this kernel: a per-thread return is safe
   const int live = hdr->live_paths;
@@ -158,6 +160,7 @@ __global__ void __launch_bounds__(kGridThreads) plan_paths_kernel(const Params P
 
 // ---- every prefix sum -------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kScanThreads) plan_scan_kernel(const Params P) {
+  ss::grid_dependency_enter();
   __shared__ int s_total_tiles;
   PlanHeader* hdr = P.hdr;
   if (block_failed(hdr)) return;
@@ -259,6 +262,7 @@ __global__ void __launch_bounds__(kScanThreads) plan_scan_kernel(const Params P)
 
 // ---- item lists ---------------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kGridThreads) plan_emit_kernel(const Params P) {
+  ss::grid_dependency_enter();
   PlanHeader* hdr = P.hdr;
   if (hdr->status != SS_OK) return;          // no barrier in this kernel
   const int live = hdr->live_paths;

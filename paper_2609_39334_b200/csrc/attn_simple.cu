@@ -89,6 +89,7 @@ __device__ void row_visit_chain(RowState& r, const Params& P, int leaf, int g, i
 
 // ---------------------------------------------------------------------------------------------------------
 __global__ void generic_kernel(const Params P) {
+  ss::grid_dependency_enter();
   if (P.hdr->status != SS_OK || P.hdr->n_generic_rows == 0) return;
   const int lane = threadIdx.x & 31;
   const int64_t warps = (static_cast<int64_t>(gridDim.x) * blockDim.x) >> 5;
@@ -117,6 +118,7 @@ __global__ void generic_kernel(const Params P) {
 }
 
 __global__ void tile_items_simple(const Params P) {
+  ss::grid_dependency_enter();
   if (P.hdr->status != SS_OK) return;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
   const int n_items = P.hdr->n_tile_items;
@@ -145,6 +147,7 @@ __global__ void tile_items_simple(const Params P) {
 }
 
 __global__ void leaf_items_simple(const Params P) {
+  ss::grid_dependency_enter();
   if (P.hdr->status != SS_OK) return;
   const int lane = threadIdx.x & 31;
   const int64_t warps = (static_cast<int64_t>(gridDim.x) * blockDim.x) >> 5;
@@ -161,6 +164,7 @@ __global__ void leaf_items_simple(const Params P) {
 
 // out = sum_s exp(lse_s - LSE) o_s,  LSE = log sum_s exp(lse_s); a token without partials (no keys) gives 0 / -inf.
 __global__ void merge_kernel(const Params P) {
+  ss::grid_dependency_enter();
   if (P.hdr->status != SS_OK) return;
   const int lane = threadIdx.x & 31;
   const int64_t warps = (static_cast<int64_t>(gridDim.x) * blockDim.x) >> 5;

@@ -28,6 +28,7 @@ __global__ void __launch_bounds__(kThreads)
 branch_sample_kernel(const float* __restrict__ logits, const int64_t* __restrict__ draw_offsets,
                      const float* __restrict__ uniforms, int vocab, double inv_temperature,
                      int32_t* __restrict__ tokens_out, int64_t* __restrict__ seq_out) {
+  ss::grid_dependency_enter();
   __shared__ double s_cdf[kChunk];
   __shared__ double s_warp[32];
   __shared__ float s_wmax[32];

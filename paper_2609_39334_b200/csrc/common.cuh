@@ -14,13 +14,33 @@ extern long long g_launch_count;
 
 inline cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
 
+// True unless the environment variable SS_NO_PDL is set (read once): launch kernels with programmatic stream
+// serialization, i.e. let a kernel's blocks become resident while the kernel before it on the stream is still
+// draining.  Every kernel of the library starts with grid_dependency_enter(), which does not return before the
+// preceding kernel has completed and its writes are visible, so the results are those of plain stream order; what
+// is saved is the launch latency between dependent kernels (several microseconds each, most of a small step).
+bool pdl_enabled();
+
 // Every kernel launch in the library goes through this macro so that launches are counted and launch errors
 // are turned into SS_ERR_CUDA.
-#define SS_LAUNCH(kernel, grid, block, smem, stream, ...)                         \
+#define SS_LAUNCH(kernel, grid_, block_, smem_, stream_, ...)                         \
   do {                                                                            \
-    kernel<<<(grid), (block), (smem), (stream)>>>(__VA_ARGS__);                   \
+    cudaLaunchConfig_t ss_cfg_ = {};                                              \
+    ss_cfg_.gridDim = dim3(static_cast<unsigned>(grid_));                          \
+    ss_cfg_.blockDim = dim3(static_cast<unsigned>(block_));                        \
+    ss_cfg_.dynamicSmemBytes = static_cast<size_t>(smem_);                        \
+    ss_cfg_.stream = (stream_);                                                   \
+    cudaLaunchAttribute ss_attr_[1];                                              \
+    ss_attr_[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;          \
+    ss_attr_[0].val.programmaticStreamSerializationAllowed = 1;                   \
+    ss_cfg_.attrs = ss_attr_;                                                     \
+    ss_cfg_.numAttrs = ::ss::pdl_enabled() ? 1 : 0;                               \
+    const cudaError_t ss_err_ = cudaLaunchKernelEx(&ss_cfg_, kernel, __VA_ARGS__); \
     ++::ss::g_launch_count;                                                       \
-    if (cudaPeekAtLastError() != cudaSuccess) { (void)cudaGetLastError(); return SS_ERR_CUDA; } \
+    if (ss_err_ != cudaSuccess || cudaPeekAtLastError() != cudaSuccess) {         \
+      (void)cudaGetLastError();                                                   \
+      return SS_ERR_CUDA;                                                         \
+    }                                                                             \
   } while (0)
 
 constexpr size_t kAlign = 256;
@@ -43,6 +63,14 @@ __host__ __device__ inline int64_t ceil_div64(int64_t a, int64_t b) { return (a 
 __host__ __device__ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
 #ifdef __CUDACC__
+// First statement of every kernel (see pdl_enabled): allow the next kernel on the stream to be scheduled early, then
+// wait until the previous kernel has completed and flushed its writes.  Both are no-ops for a kernel launched
+// without the programmatic-serialization attribute.  It must run unconditionally: a kernel that exited without
+// waiting could complete before its predecessor, and its successor would then start too early.
+__device__ __forceinline__ void grid_dependency_enter() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);

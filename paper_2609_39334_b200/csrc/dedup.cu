@@ -54,6 +54,7 @@ __device__ __forceinline__ uint32_t sort_key_of(uint64_t h, uint32_t weak) {
 __global__ void hash_kernel(const int32_t* __restrict__ tok_ids, const int64_t* __restrict__ tok_offsets,
                             const int64_t* __restrict__ ctx_key, int n, uint32_t weak, uint64_t* __restrict__ hash64,
                             uint32_t* __restrict__ keys, uint32_t* __restrict__ idx) {
+  ss::grid_dependency_enter();
   const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
   if (warp >= n) return;
@@ -67,6 +68,7 @@ __global__ void hash_kernel(const int32_t* __restrict__ tok_ids, const int64_t* 
 
 // ---- radix sort pass -------------------------------------------------------------------------------------
 __global__ void rs_hist(const uint32_t* __restrict__ keys, int n, int shift, int num_tiles, uint32_t* __restrict__ hist) {
+  ss::grid_dependency_enter();
   __shared__ uint32_t cnt[256];
   cnt[threadIdx.x] = 0;
   __syncthreads();
@@ -81,6 +83,7 @@ __global__ void rs_hist(const uint32_t* __restrict__ keys, int n, int shift, int
 
 // In-place exclusive sum scan of `count` uint32 by one block (looping with a carry).
 __global__ void scan_u32_single_block(uint32_t* __restrict__ data, int count) {
+  ss::grid_dependency_enter();
   __shared__ uint32_t warp_tot[32];
   __shared__ uint32_t carry_s;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
@@ -119,6 +122,7 @@ __global__ void scan_u32_single_block(uint32_t* __restrict__ data, int count) {
 __global__ void rs_scatter(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict__ idx_in,
                            uint32_t* __restrict__ keys_out, uint32_t* __restrict__ idx_out, int n, int shift,
                            int num_tiles, const uint32_t* __restrict__ hist) {
+  ss::grid_dependency_enter();
   __shared__ uint32_t base[256];
   __shared__ uint32_t wc[kWarpsPerSortBlock][256];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -205,6 +209,7 @@ __global__ void match_kernel(const uint32_t* __restrict__ keys, const uint32_t* 
                              const uint64_t* __restrict__ hash64, const int32_t* __restrict__ tok_ids,
                              const int64_t* __restrict__ tok_offsets, const int64_t* __restrict__ ctx_key,
                              int32_t* __restrict__ canon_out) {
+  ss::grid_dependency_enter();
   const int s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   if (s >= n) return;
   match_sorted_position(keys, idx, s, hash64, tok_ids, tok_offsets, ctx_key, canon_out, threadIdx.x & 31);
@@ -248,6 +253,7 @@ __device__ __forceinline__ void rank_block(const int32_t* canon, int n, int32_t*
 
 __global__ void rank_kernel(const int32_t* __restrict__ canon, int n, int32_t* __restrict__ rank,
                             int32_t* __restrict__ multiplicity, int32_t* __restrict__ num_unique) {
+  ss::grid_dependency_enter();
   rank_block(canon, n, rank, multiplicity, num_unique);
 }
 
@@ -266,6 +272,7 @@ __global__ void finalize_kernel(const int32_t* __restrict__ canon, const int32_t
                                 const int32_t* __restrict__ slot_in, int32_t* __restrict__ path_to_unique,
                                 int32_t* __restrict__ unique_paths, int32_t* __restrict__ multiplicity,
                                 int32_t* __restrict__ slot_out) {
+  ss::grid_dependency_enter();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n) return;
   finalize_path(canon, rank, i, slot_in, path_to_unique, unique_paths, multiplicity, slot_out);
@@ -295,6 +302,7 @@ __global__ void __launch_bounds__(kSmallThreads)
 small_hash_sort_kernel(const int32_t* __restrict__ tok_ids, const int64_t* __restrict__ tok_offsets,
                        const int64_t* __restrict__ ctx_key, int n, uint32_t weak, uint64_t* hash64, uint32_t* keys,
                        uint32_t* idx, unsigned int* counter) {
+  ss::grid_dependency_enter();
   __shared__ uint64_t skey[kSmallMax];            // (sort key << 32 | path index): distinct, so the order is total
   const int tid = threadIdx.x, lane = tid & 31;
   const int p = blockIdx.x * kSmallWarps + (tid >> 5);
@@ -333,6 +341,7 @@ small_match_finalize_kernel(const uint32_t* __restrict__ keys, const uint32_t* _
                             const int32_t* __restrict__ slot_in, int32_t* canon_out, int32_t* rank,
                             int32_t* path_to_unique, int32_t* unique_paths, int32_t* multiplicity, int32_t* slot_out,
                             int32_t* num_unique, unsigned int* counter) {
+  ss::grid_dependency_enter();
   const int s = blockIdx.x * kSmallWarps + (threadIdx.x >> 5);
   if (s < n) match_sorted_position(keys, idx, s, hash64, tok_ids, tok_offsets, ctx_key, canon_out, threadIdx.x & 31);
   if (!last_block_arrives(counter)) return;
@@ -342,7 +351,79 @@ small_match_finalize_kernel(const uint32_t* __restrict__ keys, const uint32_t* _
     finalize_path(canon_out, rank, i, slot_in, path_to_unique, unique_paths, multiplicity, slot_out);
 }
 
-__global__ void zero_scalar_kernel(int32_t* p) { *p = 0; }
+// ---- ss_gather_unique_paths ------------------------------------------------------------------------------------
+// One block.  Thread t owns kGatherItems consecutive unique paths per round: it gathers their descriptor rows and the
+// block scans the query lengths (thread sums -> warp shuffles -> warp totals -> running carry).
+constexpr int kGatherThreads = 1024;
+constexpr int kGatherItems = 4;
+
+__global__ void __launch_bounds__(kGatherThreads)
+gather_unique_kernel(const int32_t* __restrict__ unique_paths, const int32_t* __restrict__ num_unique, int n,
+                     const int32_t* __restrict__ path_leaf_node, const int32_t* __restrict__ path_q_len,
+                     const int64_t* __restrict__ q_offsets, int32_t* __restrict__ u_leaf, int32_t* __restrict__ u_q_len,
+                     int64_t* __restrict__ u_q_offsets, int64_t* __restrict__ u_q_src) {
+  ss::grid_dependency_enter();
+  __shared__ long long warp_tot[32];
+  __shared__ long long carry_s;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int U = min(max(*num_unique, 0), n);
+  if (threadIdx.x == 0) { carry_s = 0; u_q_offsets[0] = 0; }
+  __syncthreads();
+  for (int base = 0; base < n; base += kGatherThreads * kGatherItems) {
+    const int p0 = base + threadIdx.x * kGatherItems;
+    int len[kGatherItems];
+    long long mine = 0;
+#pragma unroll
+    for (int e = 0; e < kGatherItems; ++e) {
+      const int p = p0 + e;
+      len[e] = 0;
+      if (p < n) {
+        int leaf = -1;
+        long long src_row = 0;
+        if (p < U) {
+          const int src = unique_paths[p];
+          leaf = path_leaf_node[src];
+          len[e] = path_q_len[src];
+          src_row = q_offsets[src];
+        }
+        u_leaf[p] = leaf;
+        u_q_len[p] = len[e];
+        u_q_src[p] = src_row;
+      }
+      mine += len[e];
+    }
+    long long incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const long long y = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += y;
+    }
+    if (lane == 31) warp_tot[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+      long long t = warp_tot[lane];
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const long long y = __shfl_up_sync(0xffffffffu, t, o);
+        if (lane >= o) t += y;
+      }
+      warp_tot[lane] = t;
+    }
+    __syncthreads();
+    long long run = carry_s + (warp ? warp_tot[warp - 1] : 0) + incl - mine;   // rows before path p0
+#pragma unroll
+    for (int e = 0; e < kGatherItems; ++e) {
+      run += len[e];
+      if (p0 + e < n) u_q_offsets[p0 + e + 1] = run;
+    }
+    __syncthreads();
+    if (threadIdx.x == kGatherThreads - 1) carry_s = run;
+    __syncthreads();
+  }
+}
+
+__global__ void zero_scalar_kernel(int32_t* p) {
+  ss::grid_dependency_enter(); *p = 0; }
 
 struct Layout {
   size_t hash64, keys_a, keys_b, idx_a, idx_b, hist, rank, total;
@@ -502,4 +583,27 @@ extern "C" int32_t ss_dedup_paths_static(const int32_t* tok_ids, const int64_t* 
   return ss_dedup_paths(tok_ids, tok_offsets, ctx_key, slot_in, n_paths, flags, canon_out, path_to_unique_out,
                         unique_paths_out, multiplicity_out, slot_out, num_unique_out, scratch, kStaticScratchBytes,
                         stream);
+}
+
+extern "C" int32_t ss_gather_unique_paths(const int32_t* unique_paths, const int32_t* num_unique, int32_t n_paths,
+                                          const int32_t* path_leaf_node, const int32_t* path_q_len,
+                                          const int64_t* q_offsets, int32_t* u_leaf_out, int32_t* u_q_len_out,
+                                          int64_t* u_q_offsets_out, int64_t* u_q_src_out, void* stream) {
+  using namespace ss;
+  using namespace ss::dedup;
+  if (n_paths < 0 || !u_q_offsets_out) return SS_ERR_INVALID_ARG;
+  cudaStream_t st = as_stream(stream);
+  if (n_paths == 0) {
+    if (cudaMemsetAsync(u_q_offsets_out, 0, sizeof(int64_t), st) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return SS_ERR_CUDA;
+    }
+    return SS_OK;
+  }
+  if (!unique_paths || !num_unique || !path_leaf_node || !path_q_len || !q_offsets || !u_leaf_out || !u_q_len_out ||
+      !u_q_src_out)
+    return SS_ERR_INVALID_ARG;
+  SS_LAUNCH(gather_unique_kernel, 1, kGatherThreads, 0, st, unique_paths, num_unique, n_paths, path_leaf_node, path_q_len,
+            q_offsets, u_leaf_out, u_q_len_out, u_q_offsets_out, u_q_src_out);
+  return SS_OK;
 }

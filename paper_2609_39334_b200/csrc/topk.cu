@@ -43,6 +43,7 @@ __device__ void bitonic_sort(uint64_t* keys, int n_pad) {
 __global__ void __launch_bounds__(kThreads)
 topk_kernel(const float* __restrict__ scores, const int32_t* __restrict__ seg_offsets, int k,
             int32_t* __restrict__ survivors, uint8_t* __restrict__ keep, uint64_t* __restrict__ scratch) {
+  ss::grid_dependency_enter();
   __shared__ uint64_t smem_keys[kSmemKeys];
   const int s = blockIdx.x;
   const int lo = seg_offsets[s], hi = seg_offsets[s + 1];
@@ -77,6 +78,7 @@ __global__ void __launch_bounds__(kThreads)
 early_prune_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ verified,
                    const int32_t* __restrict__ seg_offsets, int k, uint8_t* __restrict__ pruned,
                    int32_t* __restrict__ selected, uint8_t* __restrict__ final_out, uint64_t* __restrict__ scratch) {
+  ss::grid_dependency_enter();
   __shared__ uint64_t smem_keys[kSmemKeys];
   __shared__ int s_nver, s_nperfect;
   const int s = blockIdx.x;

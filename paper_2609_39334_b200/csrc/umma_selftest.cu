@@ -46,6 +46,7 @@ namespace umma {
 __global__ void __launch_bounds__(128) umma_tile_test_kernel(const __grid_constant__ CUtensorMap tmap_b,
                                                              const __nv_bfloat16* __restrict__ a, float* __restrict__ c,
                                                              int n, int k, int b_mn, int32_t* status) {
+  ss::grid_dependency_enter();
   extern __shared__ __align__(1024) uint8_t smem[];
   __shared__ uint64_t bar_tma, bar_mma;
   __shared__ uint32_t tmem_slot;

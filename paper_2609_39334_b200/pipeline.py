@@ -1,9 +1,8 @@
 """Device-side plumbing around the three C-ABI calls: uploads a synthetic workload, owns the output and
-workspace tensors, and runs   ss_dedup_paths -> (gather of the unique paths) -> ss_tree_attention -> ss_topk_prune.
+workspace tensors, and runs   ss_dedup_paths -> ss_gather_unique_paths -> ss_tree_attention -> ss_topk_prune.
 
-Only memory management and argument marshalling happen here.  The one data movement that is not a library call is
-the compaction of the small per-path descriptor arrays by `unique_paths` - a plain gather that belongs to the
-caller.  The query rows themselves are not moved: the attention call reads them in place through `q_src_offsets`.
+Only memory management and argument marshalling happen here: every step is a library call.  The query rows are not
+moved by the gather: the attention call reads them in place through `q_src_offsets`.
 """
 from __future__ import annotations
 
@@ -99,21 +98,12 @@ class DevicePipeline:
                          self.canon, self.path_to_unique, self.unique_paths, self.multiplicity, self.slot_out,
                          self.num_unique, self.dedup_ws, stream=stream)
 
-    def compact_unique(self):
-        """Gather of the unique paths' descriptor rows (device-side, no host sync: entries past the live count U are
-        computed from clamped indices and ignored by the attention call).  Query rows stay where they are."""
-        N = self.N
-        if N == 0:
-            return
-        U = self.num_unique
-        ar = torch.arange(N, device=self.device)
-        live = ar < U
-        src = torch.where(live, self.unique_paths[:N].long(), torch.zeros_like(ar))
-        self.u_leaf[:N] = self.path_leaf_node[src]
-        T = torch.where(live, self.path_q_len[src].long(), torch.zeros_like(ar))
-        self.u_q_len[:N] = T.to(torch.int32)
-        self.u_q_offsets[1:] = torch.cumsum(T, 0)
-        self.u_q_src[:N] = self.q_offsets[src]
+    def compact_unique(self, stream=None):
+        """Descriptor rows of the unique paths (ss_gather_unique_paths; device-side, no host sync: entries past the
+        live count U are inert and ignored by the attention call).  Query rows stay where they are."""
+        B.ss_gather_unique_paths(self.unique_paths, self.num_unique, self.N, self.path_leaf_node, self.path_q_len,
+                                 self.q_offsets, self.u_leaf, self.u_q_len, self.u_q_offsets, self.u_q_src,
+                                 stream=stream)
 
     def attention(self, stream=None):
         B.ss_tree_attention(self.desc, self.attn_ws, stream=stream)
@@ -144,3 +134,75 @@ class DevicePipeline:
             slot_out=self.slot_out[:N].cpu().numpy(), total_q=tq,
             out=self.out[:tq].to(torch.float64).cpu().numpy(), lse=self.lse[:tq].to(torch.float64).cpu().numpy(),
             survivors=self.survivors[:self.P].cpu().numpy(), keep=self.keep[:N].cpu().numpy())
+
+
+class HostStepPipeline:
+    """`depth` independent (page-locked host buffers, device arena, stream) sets around ss_candidate_step_host, for a
+    caller whose per-step data lives in host memory.  The tree and the KV pool are those of `resident` (they stay on
+    the device).  submit(i) enqueues one whole step on set i and returns at once; alternating the sets overlaps the
+    copies of one step with the kernels of another."""
+
+    def __init__(self, resident: DevicePipeline, depth: int = 2):
+        self.resident = resident
+        w, dev = resident.w, resident.device
+        self.device = dev
+        N, P, k = w.num_paths, resident.P, w.top_k
+        Hq, D = w.num_q_heads, w.head_dim
+        tq = w.total_q
+
+        def pin(shape, dtype):
+            return torch.empty(shape, dtype=dtype, pin_memory=True)
+
+        def pin_like(a, dtype=None):
+            t = a if isinstance(a, torch.Tensor) else torch.from_numpy(np.ascontiguousarray(a))
+            out = pin(tuple(t.shape), dtype or t.dtype)
+            out.copy_(t)
+            return out
+
+        self.sets = []
+        for _ in range(depth):
+            h_in = dict(
+                tok_ids=pin_like(w.tok_ids), tok_offsets=pin_like(w.tok_offsets, torch.int64),
+                ctx_key=pin_like(w.ctx_key, torch.int64), slot_in=pin_like(w.slot_in, torch.int32),
+                path_leaf_node=pin_like(w.path_leaf_node, torch.int32), path_q_len=pin_like(w.path_q_len, torch.int32),
+                q_offsets=pin_like(w.q_offsets, torch.int64), q=pin_like(w.q),
+                scores=pin_like(w.scores, torch.float32), seg_offsets=pin_like(w.seg_offsets, torch.int32))
+            h_out = dict(
+                canon=pin((max(N, 1),), torch.int32), path_to_unique=pin((max(N, 1),), torch.int32),
+                unique_paths=pin((max(N, 1),), torch.int32), multiplicity=pin((max(N, 1),), torch.int32),
+                slot_out=pin((max(N, 1),), torch.int32), num_unique=pin((1,), torch.int32),
+                u_q_offsets=pin((N + 1,), torch.int64), out=pin((max(tq, 1), Hq, D), torch.bfloat16),
+                lse=pin((max(tq, 1), Hq), torch.float32), survivors=pin((max(P, 1), k), torch.int32),
+                keep=pin((max(N, 1),), torch.uint8), device_status=pin((1,), torch.int32))
+            step = B.make_host_step(resident.desc, n_paths=N, n_segments=P, top_k=k,
+                                    total_tok=int(w.tok_offsets[-1]), total_q=tq, host_in=h_in, host_out=h_out,
+                                    dedup_flags=resident.dedup_flags)
+            arena = B.alloc_workspace(B.ss_candidate_step_host_arena_bytes(step), dev)
+            self.sets.append(dict(h_in=h_in, h_out=h_out, step=step, arena=arena, stream=torch.cuda.Stream(dev)))
+        self.h2d_bytes = sum(t.numel() * t.element_size() for t in self.sets[0]["h_in"].values())
+        self.d2h_bytes = sum(t.numel() * t.element_size() for t in self.sets[0]["h_out"].values())
+
+    def submit(self, i: int):
+        s = self.sets[i % len(self.sets)]
+        B.ss_candidate_step_host(s["step"], s["arena"], stream=s["stream"])
+
+    def synchronize(self):
+        for s in self.sets:
+            s["stream"].synchronize()
+
+    def results(self, i: int) -> Dict[str, np.ndarray]:
+        s = self.sets[i % len(self.sets)]
+        s["stream"].synchronize()
+        o = s["h_out"]
+        st = int(o["device_status"][0])
+        if st != B.SS_OK:
+            raise B.SpecScaleError(st, "ss_candidate_step_host (device status)")
+        N, P = self.resident.N, self.resident.P
+        U = int(o["num_unique"][0])
+        tq = int(o["u_q_offsets"][U]) if N else 0
+        return dict(
+            num_unique=U, canon=o["canon"][:N].numpy().copy(), path_to_unique=o["path_to_unique"][:N].numpy().copy(),
+            unique_paths=o["unique_paths"][:U].numpy().copy(), multiplicity=o["multiplicity"][:U].numpy().copy(),
+            slot_out=o["slot_out"][:N].numpy().copy(), total_q=tq,
+            out=o["out"][:tq].to(torch.float64).numpy(), lse=o["lse"][:tq].to(torch.float64).numpy(),
+            survivors=o["survivors"][:P].numpy().copy(), keep=o["keep"][:N].numpy().copy())

@@ -102,3 +102,20 @@ def test_binding_fails_loudly_without_library(monkeypatch):
     monkeypatch.setattr(B, "LIB_PATH", "/nonexistent/libspecscale.so")
     with pytest.raises(RuntimeError, match="no CPU fallback"):
         B.lib()
+
+
+def test_every_kernel_waits_for_its_predecessor_first():
+    """Kernels are launched with programmatic stream serialization; stream order then rests on every kernel calling
+    grid_dependency_enter() before anything else (a kernel that skipped it could finish before its predecessor)."""
+    import glob
+    import re
+    csrc = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "paper_2609_39334_b200", "csrc")
+    n = 0
+    for path in sorted(glob.glob(os.path.join(csrc, "*.cu"))):
+        src = open(path).read()
+        for m in re.finditer(r"__global__[^;{]*\{", src):
+            n += 1
+            rest = src[m.end():].lstrip()
+            assert rest.startswith("ss::grid_dependency_enter();"), (os.path.basename(path), m.group(0)[:80])
+        assert "<<<" not in src, path            # every launch goes through the counting macro
+    assert n >= 20

@@ -505,3 +505,34 @@ def test_dedup_large_batch():
     assert got["num_unique"] == want["num_unique"]
     for key in ("canon", "path_to_unique", "unique_paths", "multiplicity", "slot_out"):
         assert np.array_equal(got[key], want[key]), key
+
+
+# =========================================================================================================
+# ss_gather_unique_paths
+# =========================================================================================================
+@pytest.mark.parametrize("n,frac", [(0, 0.0), (1, 1.0), (5, 0.0), (777, 0.5), (4096, 1.0), (4097, 0.9), (50000, 0.7)])
+def test_gather_unique_paths_bit_exact(n, frac):
+    dev = torch.device("cuda:0")
+    rng = np.random.default_rng(n + 3)
+    U = int(round(n * frac))
+    uniq = np.sort(rng.choice(n, size=U, replace=False)).astype(np.int32) if n else np.zeros(0, np.int32)
+    up = np.concatenate([uniq, rng.integers(0, max(n, 1), size=n - U).astype(np.int32)])
+    q_len = rng.integers(0, 130, size=n).astype(np.int32)
+    q_off = (np.concatenate([[0], np.cumsum(q_len.astype(np.int64))]) + 7).astype(np.int64)
+    leaf = rng.integers(0, 1 << 20, size=n).astype(np.int32)
+    want = oracle.gather_unique(up, U, n, leaf, q_len, q_off)
+
+    def t(a):
+        return torch.from_numpy(a).to(dev) if a.size else torch.zeros(1, dtype=torch.from_numpy(a).dtype, device=dev)
+    u_leaf = torch.full((max(n, 1),), 123, dtype=torch.int32, device=dev)
+    u_q_len = torch.full((max(n, 1),), 123, dtype=torch.int32, device=dev)
+    u_q_src = torch.full((max(n, 1),), 123, dtype=torch.int64, device=dev)
+    u_q_off = torch.full((n + 1,), 123, dtype=torch.int64, device=dev)
+    num_unique = torch.tensor([U], dtype=torch.int32, device=dev)
+    for _ in range(2):                                     # twice: no state between calls
+        B.ss_gather_unique_paths(t(up), num_unique, n, t(leaf), t(q_len), t(q_off), u_leaf, u_q_len, u_q_off, u_q_src)
+        torch.cuda.synchronize()
+        assert np.array_equal(u_leaf[:n].cpu().numpy(), want["u_leaf"])
+        assert np.array_equal(u_q_len[:n].cpu().numpy(), want["u_q_len"])
+        assert np.array_equal(u_q_src[:n].cpu().numpy(), want["u_q_src"])
+        assert np.array_equal(u_q_off.cpu().numpy(), want["u_q_offsets"])

@@ -629,3 +629,42 @@ def test_branch_sample_matches_numpy_inverse_cdf_and_frequencies():
         if pot[s] > 2000:                                 # empirical frequencies follow the softmax
             freq = np.bincount(got, minlength=V) / pot[s]
             assert np.abs(freq - p / p.sum()).max() < 0.05
+
+
+# =========================================================================================================
+# gather of the unique paths' descriptor rows
+# =========================================================================================================
+def test_gather_unique_closed_forms_and_vectorised_second_way():
+    rng = np.random.default_rng(77)
+    # all paths unique: the gather is the identity and the offsets are the input offsets
+    n = 9
+    q_len = rng.integers(1, 6, size=n).astype(np.int32)
+    q_off = np.concatenate([[0], np.cumsum(q_len)]).astype(np.int64)
+    leaf = rng.permutation(n).astype(np.int32)
+    g = oracle.gather_unique(np.arange(n, dtype=np.int32), n, n, leaf, q_len, q_off)
+    assert np.array_equal(g["u_leaf"], leaf) and np.array_equal(g["u_q_len"], q_len)
+    assert np.array_equal(g["u_q_offsets"], q_off) and np.array_equal(g["u_q_src"], q_off[:-1])
+    # worked example of the paper (three equal samples and one different -> unique paths 0 and 3)
+    g = oracle.gather_unique(np.asarray([0, 3, 0, 0], np.int32), 2, 4, np.asarray([10, 11, 12, 13], np.int32),
+                             np.asarray([1, 1, 1, 1], np.int32), np.arange(5, dtype=np.int64))
+    assert g["u_leaf"].tolist() == [10, 13, -1, -1] and g["u_q_len"].tolist() == [1, 1, 0, 0]
+    assert g["u_q_offsets"].tolist() == [0, 1, 2, 2, 2] and g["u_q_src"].tolist() == [0, 3, 0, 0]
+    # random subsets, written a second way with fancy indexing + cumsum
+    for _ in range(20):
+        n = int(rng.integers(1, 60))
+        U = int(rng.integers(0, n + 1))
+        uniq = np.sort(rng.choice(n, size=U, replace=False)).astype(np.int32)
+        up = np.concatenate([uniq, rng.integers(0, n, size=n - U).astype(np.int32)])     # garbage past U
+        q_len = rng.integers(0, 130, size=n).astype(np.int32)
+        q_off = (np.concatenate([[0], np.cumsum(q_len)]) + 5).astype(np.int64)
+        leaf = rng.integers(0, 1000, size=n).astype(np.int32)
+        g = oracle.gather_unique(up, U, n, leaf, q_len, q_off)
+        assert np.array_equal(g["u_leaf"][:U], leaf[uniq]) and np.all(g["u_leaf"][U:] == -1)
+        assert np.array_equal(g["u_q_len"][:U], q_len[uniq]) and np.all(g["u_q_len"][U:] == 0)
+        assert np.array_equal(g["u_q_src"][:U], q_off[uniq]) and np.all(g["u_q_src"][U:] == 0)
+        want = np.concatenate([[0], np.cumsum(q_len[uniq].astype(np.int64))])
+        assert np.array_equal(g["u_q_offsets"][:U + 1], want) and np.all(g["u_q_offsets"][U:] == want[-1])
+    # empty batch
+    g = oracle.gather_unique(np.zeros(0, np.int32), 0, 0, np.zeros(0, np.int32), np.zeros(0, np.int32),
+                             np.zeros(1, np.int64))
+    assert g["u_q_offsets"].tolist() == [0]
