@@ -227,6 +227,8 @@ def main():
                     help="lv-sweep: verification-attention throughput against the number of batched step tokens")
     ap.add_argument("--scale", type=float, default=1.0, help="shrink the number of problems (debugging only)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--tiles-2cta", action="store_true",
+                    help="run the tile items on the two-CTAs-per-SM kernel (64-key tiles) instead of the default one")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-depth", type=int, default=3,
                     help="independent (host buffers, device arena, stream) sets the end-to-end leg alternates between")
@@ -291,7 +293,7 @@ def main():
     # every rank its own problems: same shapes, different seed
     from paper_2609_39334_b200 import replicas
     w = replicas.replica_workload(synth.make_config, cfg_idx, rank, device=dev, scale=args.scale, poison=True)
-    pipe = DevicePipeline(w, dev)
+    pipe = DevicePipeline(w, dev, attn_flags=B.SS_FLAG_TILES_2CTA if args.tiles_2cta else 0)
     kv_bytes = pipe.kv_pool.numel() * 2
     flush = None
     if kv_bytes < 4 * L2_BYTES:
@@ -377,10 +379,11 @@ def main():
     if phase_calls["tiles"]:
         t_ms = phase_ms["tiles"] / phase_calls["tiles"]
         ach = work["tile_flops"] / (t_ms * 1e-3) / 1e12
-        roofs["tiles"] = {"kernel": "tile_items_umma_kernel", "bound": "tensor", "achieved": ach, "peak": tensor_peak,
+        roofs["tiles"] = {"kernel": "tile_items_umma_kernel" if args.tiles_2cta else "tile_items_umma_deep_kernel",
+                          "bound": "tensor", "achieved": ach, "peak": tensor_peak,
                           "unit": "TFLOP/s", "frac": ach / tensor_peak, "traffic": traffic.get("tiles"),
                           "ms_per_launch": t_ms, "peak_kind": f"{peaks['source']} {'sustained' if long_step else 'burst'}",
-                          "ctas_per_sm": int(B.lib().ss_debug_tile_kernel_occupancy())}
+                          "ctas_per_sm": 2 if args.tiles_2cta else 1}
     if phase_calls["leaves"]:
         t_ms = phase_ms["leaves"] / phase_calls["leaves"]
         ach = work["leaf_bytes"] / (t_ms * 1e-3) / 1e9

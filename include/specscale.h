@@ -51,6 +51,9 @@ extern "C" {
                                        the simple kernel instead of the tcgen05 kernel                      */
 #define SS_FLAG_WEAK_HASH 0x8u      /* dedup: truncate the path hash to 8 bits so that collisions are common;
                                        results must not change (tests the exact-comparison path)            */
+#define SS_FLAG_TILES_2CTA 0x10u    /* attention: run the tcgen05 tile items on the kernel that keeps two CTAs
+                                       per SM and works on 64-key tiles (default: the one-CTA-per-SM kernel with
+                                       128-key tiles); same results within the accuracy contract             */
 
 #define SS_MAX_DEPTH 16             /* maximum number of nodes on a root-to-leaf chain                       */
 

@@ -26,6 +26,7 @@ SS_FLAG_VALIDATE = 0x1
 SS_FLAG_FORCE_GENERIC = 0x2
 SS_FLAG_NO_TCGEN05 = 0x4
 SS_FLAG_WEAK_HASH = 0x8
+SS_FLAG_TILES_2CTA = 0x10
 SS_MAX_DEPTH = 16
 SS_DEDUP_STATIC_MAX_PATHS = 65536
 

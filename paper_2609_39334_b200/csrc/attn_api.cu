@@ -15,6 +15,7 @@ int32_t launch_leaf_items_simple(const Params& P, cudaStream_t st, int sm_count)
 int32_t launch_merge(const Params& P, cudaStream_t st, int sm_count);
 int32_t launch_leaf_items(const Params& P, cudaStream_t st, int sm_count);
 int32_t launch_tile_items_umma(const Params& P, cudaStream_t st, int sm_count);
+int32_t launch_tile_items_umma_deep(const Params& P, cudaStream_t st, int sm_count);
 
 // ---- per-phase event timing (diagnostics) ------------------------------------------------------------------
 constexpr int kProfCalls = 256;                      // timed calls between two reads
@@ -57,7 +58,7 @@ static int sm_count_of_current_device() {
 
 static int32_t check_desc(const ss_attn_desc_t* d) {
   if (!d || d->struct_size != sizeof(ss_attn_desc_t)) return SS_ERR_INVALID_ARG;
-  if (d->flags & ~(SS_FLAG_VALIDATE | SS_FLAG_FORCE_GENERIC | SS_FLAG_NO_TCGEN05)) return SS_ERR_INVALID_ARG;
+  if (d->flags & ~(SS_FLAG_VALIDATE | SS_FLAG_FORCE_GENERIC | SS_FLAG_NO_TCGEN05 | SS_FLAG_TILES_2CTA)) return SS_ERR_INVALID_ARG;
   if (d->num_q_heads < 1 || d->num_kv_heads < 1 || d->num_nodes < 0 || d->num_paths < 0 || d->total_q < 0 ||
       d->total_node_pages < 0 || d->num_pages < 0 || d->max_depth < 0 || d->max_decode_paths < 0)
     return SS_ERR_INVALID_ARG;
@@ -209,7 +210,9 @@ extern "C" int32_t ss_tree_attention(const ss_attn_desc_t* d, void* workspace, s
   ran(SS_PHASE_PLAN);
   mark(SS_PHASE_TILES);
   if (rc == SS_OK && any && !generic_only) {
-    rc = simple ? launch_tile_items_simple(P, st, sms) : launch_tile_items_umma(P, st, sms);
+    const bool two_cta = (d->flags & SS_FLAG_TILES_2CTA) != 0;
+    rc = simple ? launch_tile_items_simple(P, st, sms)
+                : (two_cta ? launch_tile_items_umma(P, st, sms) : launch_tile_items_umma_deep(P, st, sms));
     ran(SS_PHASE_TILES);
   }
   mark(SS_PHASE_LEAVES);
