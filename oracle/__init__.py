@@ -216,3 +216,64 @@ def gather_unique(unique_paths, num_unique, n_paths, path_leaf_node, path_q_len,
             u_q_src[p] = q_offsets[s]
         u_q_offsets[p + 1] = u_q_offsets[p] + int(u_q_len[p])
     return dict(u_leaf=u_leaf, u_q_len=u_q_len, u_q_offsets=u_q_offsets, u_q_src=u_q_src)
+
+
+def build_prefix_tree(tok_ids, tok_offsets, page_size=16):
+    """Radix tree of candidate paths over whole KV pages (paper, Section "Computation Deduplication": candidates share
+    25-50 % of their tokens; Section "Experimental Setup": prefix caching and sharing of KV pages).
+
+    Plain definition, written as a recursive partition: every path is cut into its full pages (tuples of `page_size`
+    token ids) and a tail (the remaining tokens).  A group of at least two paths that share more full pages than the
+    chain above them holds gets an inner node with exactly the pages ALL of them share; the group is then split
+    wherever two neighbours (in sorted order) share no further page, and every part is treated the same way.  A
+    single path gets a private leaf node with whatever the chain above it does not hold (pages + tail; possibly
+    nothing).  So only whole pages are ever shared, and every inner node has at least two children.
+    Order: paths sorted by token sequence (shorter first on a common prefix, then input index); nodes numbered in
+    depth-first preorder along that order, so parents precede children and the paths below a node are contiguous.
+
+    Returns order [n], path_leaf_node [n] (by rank), node_parent, node_kv_len, node_src_path (an input path that
+    contains the node's tokens), node_src_offset (where they start in it)."""
+    n = len(tok_offsets) - 1
+    seqs = [tuple(int(t) for t in tok_ids[tok_offsets[i]:tok_offsets[i + 1]]) for i in range(n)]
+    order = sorted(range(n), key=lambda i: (seqs[i], i))
+    pages = [tuple(seqs[i][k * page_size:(k + 1) * page_size] for k in range(len(seqs[i]) // page_size)) for i in range(n)]
+    node_parent, node_kv_len, node_src_path, node_src_offset = [], [], [], []
+    path_leaf = [0] * n
+
+    def shared_pages(a, b):                      # common full pages of two paths
+        k = 0
+        while k < len(pages[a]) and k < len(pages[b]) and pages[a][k] == pages[b][k]:
+            k += 1
+        return k
+
+    def emit(lo, hi, depth, parent):
+        """Paths order[lo:hi] all share `depth` pages, which the chain up to `parent` holds."""
+        if hi - lo == 1:
+            i = order[lo]
+            node_parent.append(parent); node_kv_len.append(len(seqs[i]) - depth * page_size)
+            node_src_path.append(i); node_src_offset.append(depth * page_size)
+            path_leaf[lo] = len(node_parent) - 1
+            return
+        common = min(shared_pages(order[lo], order[r]) for r in range(lo + 1, hi))
+        if common > depth:                        # an inner node with the pages every path of the group shares
+            node_parent.append(parent); node_kv_len.append((common - depth) * page_size)
+            node_src_path.append(order[lo]); node_src_offset.append(depth * page_size)
+            parent = len(node_parent) - 1
+            depth = common
+        # split where neighbours share no more than `depth` pages
+        start = lo
+        for r in range(lo + 1, hi + 1):
+            if r == hi or shared_pages(order[r - 1], order[r]) <= depth:
+                emit(start, r, depth, parent)
+                start = r
+
+    if n:
+        # top level: groups of neighbours that share at least one page; single paths otherwise
+        start = 0
+        for r in range(1, n + 1):
+            if r == n or shared_pages(order[r - 1], order[r]) == 0:
+                emit(start, r, 0, -1)
+                start = r
+    return dict(order=np.asarray(order, np.int32), path_leaf_node=np.asarray(path_leaf, np.int32),
+                node_parent=np.asarray(node_parent, np.int32), node_kv_len=np.asarray(node_kv_len, np.int32),
+                node_src_path=np.asarray(node_src_path, np.int32), node_src_offset=np.asarray(node_src_offset, np.int32))

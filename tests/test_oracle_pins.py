@@ -668,3 +668,101 @@ def test_gather_unique_closed_forms_and_vectorised_second_way():
     g = oracle.gather_unique(np.zeros(0, np.int32), 0, 0, np.zeros(0, np.int32), np.zeros(0, np.int32),
                              np.zeros(1, np.int64))
     assert g["u_q_offsets"].tolist() == [0]
+
+
+# =========================================================================================================
+# radix tree over whole pages
+# =========================================================================================================
+def check_prefix_tree_invariants(seqs, t, page):
+    """Properties that characterise the tree, checked without the oracle's algorithm."""
+    n = len(seqs)
+    order, leaf = t["order"], t["path_leaf_node"]
+    parent, kv, sp, so = t["node_parent"], t["node_kv_len"], t["node_src_path"], t["node_src_offset"]
+    assert sorted(order.tolist()) == list(range(n))
+    keys = [(tuple(seqs[i]), i) for i in order]
+    assert keys == sorted(keys)                                        # lexicographic, ties by index
+    assert all(parent[v] < v for v in range(len(parent)))              # parents precede children
+    below = [[] for _ in parent]
+    for r in range(n):
+        # the chain root -> leaf spells the path
+        chain, v = [], int(leaf[r])
+        while v >= 0:
+            chain.append(v); v = int(parent[v])
+        toks = []
+        for v in reversed(chain):
+            assert so[v] == len(toks)                                  # a node starts where the chain above it ends
+            toks += list(seqs[sp[v]][so[v]:so[v] + kv[v]])
+            below[v].append(r)
+        assert toks == list(seqs[order[r]])
+    children = [[] for _ in parent]
+    for v in range(len(parent)):
+        if parent[v] >= 0:
+            children[parent[v]].append(v)
+    n_inner = 0
+    for v in range(len(parent)):
+        b = below[v]
+        assert b == list(range(b[0], b[-1] + 1))                       # the paths below a node are contiguous
+        if len(b) > 1:
+            n_inner += 1
+            assert kv[v] % page == 0 and kv[v] > 0                     # shared nodes hold whole pages
+            assert len(children[v]) >= 2                               # ... and branch
+    assert n_inner + n == len(parent)                                  # everything else is a private leaf
+    # maximality: two children of one parent (or two roots) never start with the same full page
+    groups = {}
+    for v in range(len(parent)):
+        groups.setdefault(int(parent[v]), []).append(v)
+    for vs in groups.values():
+        firsts = [tuple(seqs[order[below[v][0]]][so[v]:so[v] + page]) for v in vs
+                  if len(seqs[order[below[v][0]]]) - so[v] >= page]
+        assert len(firsts) == len(set(firsts))
+
+
+def test_prefix_tree_hand_worked_example():
+    want = {}
+    for line in open(os.path.join(GOLDEN, "prefix_tree_example.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        k, *v = line.split()
+        want[k] = [int(x) for x in v]
+    seqs = [[1, 2, 3, 4, 5, 6, 7, 8, 9], [1, 2, 3, 4, 5, 6, 7, 8, 10, 11], [1, 2, 3, 4, 9, 9, 9, 9], [7],
+            [1, 2, 3, 4, 5, 6, 7, 8], []]
+    ids, off = csr(seqs)
+    t = oracle.build_prefix_tree(ids, off, want["page_size"][0])
+    for k in ("order", "path_leaf_node", "node_parent", "node_kv_len", "node_src_offset"):
+        assert t[k].tolist() == want[k], k
+    check_prefix_tree_invariants(seqs, t, 4)
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_prefix_tree_invariants_on_random_trees(seed):
+    """Sequences drawn from a random tree with known sharing: the oracle's tree must spell every path, share whole
+    pages only, be maximal, and share exactly as many tokens as the generating tree does."""
+    rng = np.random.default_rng(seed)
+    page = int(rng.choice([2, 4, 16]))
+    seqs = []
+
+    def grow(prefix, depth):
+        fan = int(rng.integers(1, 4)) if depth < 3 else 1
+        for _ in range(fan):
+            if depth < 3 and rng.random() < 0.6:
+                seg = [int(x) for x in rng.integers(0, 3, size=page * int(rng.integers(1, 3)))]
+                grow(prefix + seg, depth + 1)
+            else:
+                seqs.append(prefix + [int(x) for x in rng.integers(0, 3, size=int(rng.integers(0, 2 * page)))])
+
+    grow([], 0)
+    perm = rng.permutation(len(seqs))
+    seqs = [seqs[i] for i in perm]
+    ids, off = csr(seqs)
+    t = oracle.build_prefix_tree(ids, off, page)
+    check_prefix_tree_invariants(seqs, t, page)
+    # tokens stored = sum over sorted neighbours of what is NOT shared in whole pages (brute force, second way)
+    order = t["order"]
+    stored = len(seqs[order[0]]) if len(seqs) else 0
+    for r in range(1, len(seqs)):
+        a, b = seqs[order[r - 1]], seqs[order[r]]
+        k = 0
+        while k < len(a) and k < len(b) and a[k] == b[k]:
+            k += 1
+        stored += len(b) - (k // page) * page
+    assert int(t["node_kv_len"].sum()) == stored
