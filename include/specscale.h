@@ -309,6 +309,45 @@ int32_t ss_branch_sample(const float* logits, const int64_t* draw_offsets, const
                          int32_t vocab, float temperature, int32_t* tokens_out, int64_t* seq_out, void* stream);
 
 /* =========================================================================================================
+ * ss_build_prefix_tree - radix tree of candidate paths over whole KV pages, from raw token ids.
+ *
+ * Paper: Section "Computation Deduplication" (a quarter to a half of the tokens that the candidates of a step
+ * generate are common across candidates) and Section "Experimental Setup" (prefix KV caching and sharing):
+ * beyond removing candidates that are equal as a whole (ss_dedup_paths), candidates that agree on a prefix can keep
+ * that prefix's KV once.  This call finds the sharing: it returns the tree (parents before children) in exactly the
+ * form ss_tree_attention takes, with only WHOLE pages shared, so that a node's pages can be the physical pages of
+ * any path below it.
+ *
+ * Definition (unique): paths are ordered by token sequence (a proper prefix first, then the input index).  A group
+ * of at least two neighbouring paths that share more full pages than the chain above them holds gets an inner node
+ * with exactly the pages all of them share; the group splits where two neighbours share no further page; a single
+ * path gets a private leaf node with whatever the chain above it does not hold (possibly nothing).  Nodes are
+ * numbered depth-first along the order, so the paths below a node are contiguous.
+ *
+ *   tok_ids, tok_offsets  as in ss_dedup_paths, with tok_offsets[0] == 0
+ *   n_paths               host, 0 .. SS_PREFIX_TREE_MAX_PATHS;  total_tok  host, >= tok_offsets[n_paths]
+ *   page_size             host, >= 1 (16 for ss_tree_attention)
+ *   order_out           int32 [n_paths]     input index of the path of every rank
+ *   path_leaf_node_out  int32 [n_paths]     by rank
+ *   node_parent_out, node_kv_len_out                int32 [2*n_paths]   first *num_nodes_out entries valid
+ *   node_src_path_out, node_src_offset_out          int32 [2*n_paths]   an input path that contains the node's tokens
+ *                                                                        and the position where they start in it
+ *   num_nodes_out       int32 [1]           n_paths leaves + the inner nodes (0 after a device-side error)
+ *   workspace           >= ss_prefix_tree_workspace_bytes(...) bytes, 256-byte aligned; its first word is the device
+ *                       status (ss_last_device_status): SS_ERR_BAD_INPUT if the internal 64-bit page hashes collided
+ *                       in a way that mis-ordered two paths (the tree is then withheld, never wrong)
+ * Errors (host): SS_ERR_INVALID_ARG, SS_ERR_WORKSPACE_TOO_SMALL, SS_ERR_CUDA.
+ * ======================================================================================================= */
+#define SS_PREFIX_TREE_MAX_PATHS (1 << 20)
+int32_t ss_prefix_tree_workspace_bytes(int32_t n_paths, int64_t total_tok, int32_t page_size,
+                                       size_t* out_bytes /* host */);
+int32_t ss_build_prefix_tree(const int32_t* tok_ids, const int64_t* tok_offsets, int32_t n_paths, int64_t total_tok,
+                             int32_t page_size, int32_t* order_out, int32_t* path_leaf_node_out,
+                             int32_t* node_parent_out, int32_t* node_kv_len_out, int32_t* node_src_path_out,
+                             int32_t* node_src_offset_out, int32_t* num_nodes_out, void* workspace,
+                             size_t workspace_bytes, void* stream);
+
+/* =========================================================================================================
  * ss_candidate_step_host - one pass of the whole path for per-step data that lives in HOST memory.
  *
  * Paper: the system overview figure and Sections "Computation Deduplication", "Lazy Verification" and "Early

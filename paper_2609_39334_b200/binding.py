@@ -36,6 +36,7 @@ EXPORTS = [
     "ss_launch_count", "ss_debug_umma_tile", "ss_profile_enable", "ss_profile_read",
     "ss_dedup_paths_static", "ss_debug_tile_kernel_occupancy", "ss_early_prune",
     "ss_branch_sample", "ss_gather_unique_paths", "ss_candidate_step_host_arena_bytes", "ss_candidate_step_host",
+    "ss_prefix_tree_workspace_bytes", "ss_build_prefix_tree",
 ]
 PHASES = ["plan", "tiles", "leaves", "generic", "merge"]
 
@@ -168,6 +169,28 @@ def ss_gather_unique_paths(unique_paths, num_unique, n_paths, path_leaf_node, pa
                                       _ptr(u_q_len_out), _ptr(u_q_offsets_out), _ptr(u_q_src_out), _stream(stream))
     if check:
         _check(rc, "ss_gather_unique_paths")
+    return rc
+
+
+def ss_prefix_tree_workspace_bytes(n_paths: int, total_tok: int, page_size: int = 16) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().ss_prefix_tree_workspace_bytes(ctypes.c_int32(n_paths), ctypes.c_int64(total_tok),
+                                                ctypes.c_int32(page_size), ctypes.byref(out)),
+           "ss_prefix_tree_workspace_bytes")
+    return int(out.value)
+
+
+def ss_build_prefix_tree(tok_ids, tok_offsets, n_paths, total_tok, page_size, order_out, path_leaf_node_out,
+                         node_parent_out, node_kv_len_out, node_src_path_out, node_src_offset_out, num_nodes_out,
+                         workspace, stream=None, check=True) -> int:
+    """Radix tree of the paths over whole pages (parents before children, paths in sorted order)."""
+    rc = lib().ss_build_prefix_tree(_ptr(tok_ids), _ptr(tok_offsets), ctypes.c_int32(n_paths), ctypes.c_int64(total_tok),
+                                    ctypes.c_int32(page_size), _ptr(order_out), _ptr(path_leaf_node_out),
+                                    _ptr(node_parent_out), _ptr(node_kv_len_out), _ptr(node_src_path_out),
+                                    _ptr(node_src_offset_out), _ptr(num_nodes_out), _ptr(workspace),
+                                    ctypes.c_size_t(workspace.numel() * workspace.element_size()), _stream(stream))
+    if check:
+        _check(rc, "ss_build_prefix_tree")
     return rc
 
 
