@@ -229,6 +229,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--tiles-2cta", action="store_true",
                     help="run the tile items on the two-CTAs-per-SM kernel (64-key tiles) instead of the default one")
+    ap.add_argument("--graph", action="store_true",
+                    help="also time the step as a CUDA graph replay (reported as ms_per_step_cuda_graph)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-depth", type=int, default=3,
                     help="independent (host buffers, device arena, stream) sets the end-to-end leg alternates between")
@@ -348,6 +350,29 @@ def main():
         pipe.step()
         ev2[i][1].record()
     sync_all()
+    # optionally once more as a CUDA graph replay (one graph = one whole step): what a serving loop that calls the same
+    # step shape repeatedly would pay; every call of the library is stream-ordered and allocation-free, so it captures
+    graph_ms = None
+    if args.graph:
+        side = torch.cuda.Stream(dev)
+        side.wait_stream(torch.cuda.current_stream(dev))
+        with torch.cuda.stream(side):
+            pipe.step()                                   # first-use initialisation outside the capture
+        torch.cuda.current_stream(dev).wait_stream(side)
+        sync_all()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            pipe.step()
+        ev3 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+        sync_all()
+        for i in range(args.steps):
+            if flush is not None:
+                flush.fill_(i & 0xff)
+            ev3[i][0].record()
+            g.replay()
+            ev3[i][1].record()
+        sync_all()
+        graph_ms = replicas.max_over_ranks(float(sum(a.elapsed_time(b) for a, b in ev3)), dev) / args.steps
     clk = clocks.stop() if rank == 0 else None
     plain_ms = replicas.max_over_ranks(float(sum(a.elapsed_time(b) for a, b in ev2)), dev) / args.steps
     step_ms = [a.elapsed_time(b) for a, b in ev]
@@ -405,6 +430,7 @@ def main():
         "attention_ms_per_step": attn_ms,
         "attention_tokens_per_s": world * tokens / (attn_ms * 1e-3) if attn_ms > 0 else None,
         "ms_per_step_without_phase_events": plain_ms,
+        "ms_per_step_cuda_graph": graph_ms,
         "phase_ms_per_step": {k: (phase_ms[k] / phase_calls[k] if phase_calls[k] else 0.0) for k in phase_ms},
         "roofline": roofs.get(dominant) if dominant else None,
         "roofline_phases": roofs,
