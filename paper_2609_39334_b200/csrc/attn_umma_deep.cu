@@ -214,6 +214,9 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
         mbar_arrive(&C.q_full);
         int limit_row = (it.kind == kItemChain) ? it.limit0 + i : it.limit0;
         if (limit_row > it.kv_end) limit_row = it.kv_end;
+        // first tile in which some row of this warp has a masked column (causal tail / end of the source): tiles
+        // before it need neither the mask nor a vote about it
+        const int first_masked_tile = __reduce_min_sync(0xffffffffu, max(limit_row - it.kv_begin, 0) / kTile);
         for (int j = 0; j < n_tiles; ++j) {
           const uint32_t gj = g_tile + j;
           const int b = gj % kRing;
@@ -222,15 +225,21 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           tc_fence_after();
+          // the second half of the scores is fetched while the exponentials of the first half are computed
           uint32_t sr[kTile];
-#pragma unroll
-          for (int c0 = 0; c0 < kTile; c0 += 32)
-            tmem_ld32(tmem + lane_base + s_col + c0, *reinterpret_cast<uint32_t(*)[32]>(&sr[c0]));
+          tmem_ld32(tmem + lane_base + s_col, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
+          tmem_ld32(tmem + lane_base + s_col + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
           tmem_wait_ld();
+          tmem_ld32(tmem + lane_base + s_col + 64, *reinterpret_cast<uint32_t(*)[32]>(&sr[64]));
+          tmem_ld32(tmem + lane_base + s_col + 96, *reinterpret_cast<uint32_t(*)[32]>(&sr[96]));
 
           const int pos0 = it.kv_begin + j * kTile;
-          const int nvis = limit_row - pos0;                      // visible columns of this tile for this row
-          if (!__all_sync(0xffffffffu, nvis >= kTile)) {          // causal tail or end of the source: mask
+          const bool masked = j >= first_masked_tile;             // warp-uniform
+          if (masked) {                                           // causal tail or end of the source
+            tmem_wait_ld();
+            tmem_pin32(*reinterpret_cast<uint32_t(*)[32]>(&sr[64]));
+            tmem_pin32(*reinterpret_cast<uint32_t(*)[32]>(&sr[96]));
+            const int nvis = limit_row - pos0;                    // visible columns of this tile for this row
 #pragma unroll
             for (int c = 0; c < kTile; ++c)
               if (c >= nvis) sr[c] = 0xff800000u;                 // -inf
@@ -257,14 +266,22 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
           float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
           uint32_t pr[kTile / 2];
 #pragma unroll
-          for (int c = 0; c < kTile; c += 2) {
-            const float s0 = __uint_as_float(sr[c]), s1 = __uint_as_float(sr[c + 1]);
-            float x0, x1;
-            unpack2(fma2(pack2(s0, s1), cl2_2, nmc2), x0, x1);
-            const float p0 = ex2(x0), p1 = ex2(x1);
-            sum2[(c >> 1) & 1] = add2(sum2[(c >> 1) & 1], pack2(p0, p1));
-            pr[c >> 1] = pack_bf16_rn(p0, p1);
-            if ((c & 6) == 0) mx4[(c >> 3) & 3] = max3(mx4[(c >> 3) & 3], s0, s1);   // every fourth pair
+          for (int hf = 0; hf < 2; ++hf) {
+            if (hf == 1) {
+              tmem_wait_ld();                                     // (no-op when the mask path has waited already)
+              tmem_pin32(*reinterpret_cast<uint32_t(*)[32]>(&sr[64]));
+              tmem_pin32(*reinterpret_cast<uint32_t(*)[32]>(&sr[96]));
+            }
+#pragma unroll
+            for (int c = hf * 64; c < hf * 64 + 64; c += 2) {
+              const float s0 = __uint_as_float(sr[c]), s1 = __uint_as_float(sr[c + 1]);
+              float x0, x1;
+              unpack2(fma2(pack2(s0, s1), cl2_2, nmc2), x0, x1);
+              const float p0 = ex2(x0), p1 = ex2(x1);
+              sum2[(c >> 1) & 1] = add2(sum2[(c >> 1) & 1], pack2(p0, p1));
+              pr[c >> 1] = pack_bf16_rn(p0, p1);
+              if ((c & 6) == 0) mx4[(c >> 3) & 3] = max3(mx4[(c >> 3) & 3], s0, s1);   // every fourth pair
+            }
           }
           float sum4[4];
           unpack2(sum2[0], sum4[0], sum4[1]);
@@ -274,7 +291,10 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
           float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
           const float tile_sum = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
           const bool jump = m == -INFINITY || !(tile_sum <= jump_sum);   // no reference yet, or beyond 2^kJumpLog2 / inf / NaN
-          if (__any_sync(0xffffffffu, jump)) {
+          const int n_keys = min(kTile, it.kv_end - pos0);
+          // one vote covers every rare path of a tile: exact fallback, O rescale, ragged end of the source
+          const bool rare = __any_sync(0xffffffffu, jump || (alpha != 1.f && j > 0)) || n_keys < kTile;
+          if (rare && __any_sync(0xffffffffu, jump)) {
             if (jump) {                                           // exact path: this tile's own maximum is the reference
 #pragma unroll
               for (int c = 0; c < kTile; c += 2)
@@ -301,7 +321,7 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
           m_next = mx > m + lazy_raw ? mx : m;
           const bool move = alpha != 1.f;
 
-          if (__any_sync(0xffffffffu, move && j > 0)) {           // rescale O (warp-collective TMEM access)
+          if (rare && __any_sync(0xffffffffu, move && j > 0)) {   // rescale O (warp-collective TMEM access)
             ok = mbar_wait(&C.pv_done[(gj - 1) % kRing], ((gj - 1) / kRing) & 1, abort_flag);   // PV(j-1) has landed in O
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
@@ -318,7 +338,6 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
             tmem_wait_st();
           }
           // ---- last tile of a source that ends inside a page / inside the tile: zero the V rows past the end ---
-          const int n_keys = min(kTile, it.kv_end - pos0);
           if (n_keys < kTile) {
             const int s = gj % kStagesV;
             ok = mbar_wait(&C.v_full[s], (gj / kStagesV) & 1, abort_flag);
