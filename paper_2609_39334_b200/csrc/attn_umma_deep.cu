@@ -257,6 +257,17 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
             m = m_next;
             l *= alpha;
           }
+          if (j == 0) {                                           // no reference yet: take this tile's exact maximum first
+            tmem_wait_ld();                                       // (instead of exponentials that the fallback would redo)
+            tmem_pin32(*reinterpret_cast<uint32_t(*)[32]>(&sr[64]));
+            tmem_pin32(*reinterpret_cast<uint32_t(*)[32]>(&sr[96]));
+            float e4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+            for (int c = 0; c < kTile; c += 2)
+              e4[(c >> 1) & 3] = max3(e4[(c >> 1) & 3], __uint_as_float(sr[c]), __uint_as_float(sr[c + 1]));
+            const float mxe = fmaxf(fmaxf(e4[0], e4[1]), fmaxf(e4[2], e4[3]));
+            if (mxe > -INFINITY) { m = mxe; m_next = mxe; }
+          }
           float mc = m == -INFINITY ? 0.f : m * cl2;
           // Every instruction of this loop costs an issue slot that the SFU does not hide (an ex2 holds the
           // sub-partition for 8 clocks and the rest adds to it), so the scaling and the row sum work on fp32 pairs.
