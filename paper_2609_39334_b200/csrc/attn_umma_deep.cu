@@ -46,7 +46,7 @@ constexpr int kUmmaSmem = kOffV + kStagesV * kStageBytes;   // + the control blo
 struct Ctrl {
   // All per-buffer barriers are indexed by tile number modulo the ring / stage count and waited with the parity of
   // (tile number / count); a waiter is never two completions away from its barrier (see the role loops).
-  uint64_t q_full, k_full[kStagesK], v_full[kStagesV], k_empty[kStagesK], v_empty[kStagesV], s_full[kRing],
+  uint64_t q_full, q_full_tma, k_full[kStagesK], v_full[kStagesV], k_empty[kStagesK], v_empty[kStagesV], s_full[kRing],
       p_full[kRing], pv_done[kRing], o_final, item_ready[2];
   uint32_t tmem_slot;
   int abort_flag;
@@ -94,7 +94,7 @@ __device__ __forceinline__ ItemView view(const TileItem& it) {
 
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
-                       const Params P) {
+                            const __grid_constant__ CUtensorMap tmap_q, const Params P) {
   ss::grid_dependency_enter();
   extern __shared__ __align__(1024) uint8_t smem[];
   __shared__ Ctrl C;
@@ -103,7 +103,8 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
 
   if (tid == 0) {
     C.abort_flag = (smem_u32(smem) & 1023u) ? 1 : 0;
-    mbar_init(&C.q_full, kSoftmaxWarps * 32);
+    mbar_init(&C.q_full, kSoftmaxWarps * 32);       // stacked items: the softmax threads copy the (gathered) rows
+    mbar_init(&C.q_full_tma, 1);                    // chain items: one TMA box pair
     for (int s = 0; s < kStagesK; ++s) { mbar_init(&C.k_full[s], 1); mbar_init(&C.k_empty[s], 1); }
     for (int s = 0; s < kStagesV; ++s) { mbar_init(&C.v_full[s], 1); mbar_init(&C.v_empty[s], 1); }
     mbar_init(&C.item_ready[0], 1);
@@ -115,7 +116,10 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
     fence_barrier_init();
     prefetch_tensormap(&tmap_k);
     prefetch_tensormap(&tmap_v);
+    prefetch_tensormap(&tmap_q);
   }
+  for (int x = tid; x < 65536 / 16; x += kUmmaThreads) reinterpret_cast<uint4*>(smem + kOffQ)[x] = make_uint4(0, 0, 0, 0);
+  fence_proxy_async_smem();
   if (warp == kSoftmaxWarps) tmem_alloc(&C.tmem_slot, kTmemCols);
   tc_fence_before();
   __syncthreads();
@@ -129,6 +133,7 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
 
   uint32_t g_tile = 0;      // tiles this CTA has processed (identical in every role)
   uint32_t q_uses = 0;      // items with at least one tile
+  uint32_t q_uses_tma = 0;  // ... of them chain items (their Q arrives through TMA and q_full_tma)
   uint32_t item_seq = 0;    // items this CTA has started
   int n_prefetched = 0;     // producer warps: tiles of the current item that were issued during the previous one
 
@@ -159,6 +164,16 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
     asm volatile("cp.async.commit_group;" ::: "memory");
   };
 
+  // Chain items: the Q rows are tokens [src0, src0 + tokens per tile) x the G heads of the group x 128 dims, a box of
+  // the query tensor (one thread; rows of the box past the item's tokens belong to other paths or are zero-filled:
+  // finite either way, and never written out).
+  auto q_tma_start = [&](const ItemView& v, int buf) {
+    uint8_t* dst = smem + kOffQ + buf * 32768;
+    mbar_arrive_expect_tx(&C.q_full_tma, static_cast<uint32_t>(2 * 128 * G * P.tok_per_tile));
+    tma_load_3d(dst, &tmap_q, 0, v.g * G, v.src0, &C.q_full_tma);
+    tma_load_3d(dst + 16384, &tmap_q, 64, v.g * G, v.src0, &C.q_full_tma);
+  };
+
   if (tid == 0) fetch_item(0);
   __syncthreads();
   if (warp < kSoftmaxWarps) {                                    // Q of the first item
@@ -166,8 +181,16 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
       const int e0 = C.item_e[0];
       if (e0 >= 0 && e0 < n_items) {
         const ItemView v0 = view(C.item[0]);
-        if (v0.n_tiles > 0) q_copy_start(v0, 0);
+        if (v0.n_tiles > 0 && v0.kind != kItemChain) q_copy_start(v0, 0);
       }
+    }
+  }
+
+  if (tid == kSoftmaxWarps * 32 && mbar_wait(&C.item_ready[0], 0, abort_flag)) {   // K producer: Q of a first chain item
+    const int e0 = C.item_e[0];
+    if (e0 >= 0 && e0 < n_items) {
+      const ItemView v0 = view(C.item[0]);
+      if (v0.n_tiles > 0 && v0.kind == kItemChain) q_tma_start(v0, 0);
     }
   }
 
@@ -204,14 +227,17 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
         const int e_next = C.item_e[slot ^ 1];
         if (e_next < 0 || e_next >= n_items) return;
         const ItemView nv = view(C.item[slot ^ 1]);
-        if (nv.n_tiles > 0) q_copy_start(nv, slot ^ 1);
+        if (nv.n_tiles > 0 && nv.kind != kItemChain) q_copy_start(nv, slot ^ 1);
       };
       if (n_tiles == 0) start_next_q();
       if (n_tiles > 0) {
-        // ---- Q rows of this item: their asynchronous copy was started during the previous item -----------------------
-        asm volatile("cp.async.wait_group 0;" ::: "memory");
-        fence_proxy_async_smem();
-        mbar_arrive(&C.q_full);
+        // ---- Q rows of a stacked item: their asynchronous copy was started during the previous item (a chain item's
+        //      rows come through TMA, issued by the K producer) --------------------------------------------------------
+        if (it.kind != kItemChain) {
+          asm volatile("cp.async.wait_group 0;" ::: "memory");
+          fence_proxy_async_smem();
+          mbar_arrive(&C.q_full);
+        }
         int limit_row = (it.kind == kItemChain) ? it.limit0 + i : it.limit0;
         if (limit_row > it.kv_end) limit_row = it.kv_end;
         // first tile in which some row of this warp has a masked column (causal tail / end of the source): tiles
@@ -517,6 +543,8 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
         if (e_next >= 0 && e_next < n_items) {
           const ItemView nv = view(C.item[slot ^ 1]);
           n_prefetched = min(nv.n_tiles, n_stages);
+          // Q buffer slot ^ 1 is free: the products of the item before this one have completed
+          if (which == 0 && lane == 0 && nv.n_tiles > 0 && nv.kind == kItemChain) q_tma_start(nv, slot ^ 1);
           if (!stream_tiles(nv, g_tile + n_tiles, 0, n_prefetched)) n_prefetched = 0;   // (aborting)
         }
       }
@@ -526,7 +554,8 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
         constexpr uint32_t idesc_qk = instr_desc_bf16(128, kTile, false);
         const uint64_t q_desc0 = smem_desc_sw128(smem_u32(smem + kOffQ + slot * 32768), 0, 1024);
         const uint64_t k_desc0 = smem_desc_sw128(smem_u32(smem + kOffK), 0, 1024);
-        bool ok = mbar_wait(&C.q_full, q_uses & 1, abort_flag);
+        bool ok = it.kind == kItemChain ? mbar_wait(&C.q_full_tma, q_uses_tma & 1, abort_flag)
+                                        : mbar_wait(&C.q_full, (q_uses - q_uses_tma) & 1, abort_flag);
         for (int j = 0; j < n_tiles && ok; ++j) {
           const uint32_t gj = g_tile + j;
           const int s = gj % kStagesK, b = gj % kRing;
@@ -576,7 +605,10 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
     __syncthreads();
     tc_fence_after();
     g_tile += n_tiles;
-    if (n_tiles > 0) ++q_uses;
+    if (n_tiles > 0) {
+      ++q_uses;
+      if (it.kind == kItemChain) ++q_uses_tma;
+    }
     ++item_seq;
   }
 
@@ -611,7 +643,12 @@ int32_t launch_tile_items_umma_deep(const Params& P, cudaStream_t st, int sm_cou
       !tmap::encode_2d_bf16(&tv, P.v_pool, kHeadDim, static_cast<uint64_t>(rows), kHeadDim * 2, kPage))
     return SS_ERR_CUDA;
   // one CTA per SM: the kernel takes all 512 TMEM columns and most of the shared memory
-  SS_LAUNCH(tile_items_umma_deep_kernel, sm_count, kUmmaThreads, kUmmaSmem, st, tk, tv, P);
+  CUtensorMap tq;
+  const int64_t q_rows = P.q_src_offsets ? P.q_src_rows : P.total_q;
+  if (!tmap::encode_q_bf16(&tq, P.q, static_cast<uint64_t>(P.Hq), static_cast<uint64_t>(q_rows > 0 ? q_rows : 1),
+                           static_cast<uint32_t>(P.G), static_cast<uint32_t>(P.tok_per_tile)))
+    return SS_ERR_CUDA;
+  SS_LAUNCH(tile_items_umma_deep_kernel, sm_count, kUmmaThreads, kUmmaSmem, st, tk, tv, tq, P);
   return SS_OK;
 }
 

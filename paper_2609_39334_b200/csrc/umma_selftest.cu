@@ -39,6 +39,21 @@ bool encode_2d_bf16(CUtensorMap* out, const void* base, uint64_t row_elems, uint
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Query rows: q viewed as [token][q head][128] bf16; boxes of 64 dims x `heads` heads x `tokens` tokens land in shared
+// memory as consecutive 128-byte rows (token-major, then head) with the 128-byte swizzle.
+bool encode_q_bf16(CUtensorMap* out, const void* base, uint64_t q_heads, uint64_t tokens_total, uint32_t heads,
+                   uint32_t tokens) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[3] = {128, q_heads, tokens_total};
+  const cuuint64_t strides[2] = {256, q_heads * 256};
+  const cuuint32_t box[3] = {64, heads, tokens};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace tmap
 
 namespace umma {
