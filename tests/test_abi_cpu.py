@@ -119,3 +119,20 @@ def test_every_kernel_waits_for_its_predecessor_first():
             assert rest.startswith("ss::grid_dependency_enter();"), (os.path.basename(path), m.group(0)[:80])
         assert "<<<" not in src, path            # every launch goes through the counting macro
     assert n >= 20
+
+
+def test_profiles_carry_the_dram_traffic_the_bench_reports():
+    """bench.py fills roofline.traffic from profiles/dram_traffic.txt; the file must hold a figure for both attention
+    kernels of the timed workload, and every summary beside it must state the command that made it."""
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    rows = {}
+    with open(os.path.join(root, "profiles", "dram_traffic.txt")) as f:
+        for line in f:
+            parts = line.split()
+            if len(parts) == 3 and not line.startswith("#"):
+                rows[(parts[0], parts[1])] = float(parts[2])
+    assert rows.get(("c5", "tiles"), 0) > 1e9 and rows.get(("c5", "leaves"), 0) > 1e9
+    for name in os.listdir(os.path.join(root, "profiles")):
+        if name.endswith(".md"):
+            with open(os.path.join(root, "profiles", name)) as f:
+                assert "ncu " in f.read(), name
