@@ -30,6 +30,8 @@ UNIT = "tokens/s"
 WORKLOADS = {"c2": 2, "c3": 3, "c4": 4, "c5": 5}
 LV_SWEEP_TOKENS = [256, 512, 1024, 2048, 4096, 8192, 16384]
 L2_BYTES = 126 * 1024 * 1024
+NOMINAL_HBM_GBS = 8000.0            # vendor figures, reported beside the measured peaks for context only
+NOMINAL_BF16_TFLOPS = 2250.0
 
 
 def load_peaks():
@@ -408,13 +410,15 @@ def main():
                           "bound": "tensor", "achieved": ach, "peak": tensor_peak,
                           "unit": "TFLOP/s", "frac": ach / tensor_peak, "traffic": traffic.get("tiles"),
                           "ms_per_launch": t_ms, "peak_kind": f"{peaks['source']} {'sustained' if long_step else 'burst'}",
+                          "frac_of_nominal": ach / NOMINAL_BF16_TFLOPS, "nominal_peak": NOMINAL_BF16_TFLOPS,
                           "ctas_per_sm": 2 if args.tiles_2cta else 1}
     if phase_calls["leaves"]:
         t_ms = phase_ms["leaves"] / phase_calls["leaves"]
         ach = work["leaf_bytes"] / (t_ms * 1e-3) / 1e9
         roofs["leaves"] = {"kernel": "leaf_items_kernel", "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"],
                            "unit": "GB/s", "frac": ach / peaks["hbm_gbs"], "traffic": traffic.get("leaves"),
-                           "ms_per_launch": t_ms, "peak_kind": f"{peaks['source']} copy"}
+                           "ms_per_launch": t_ms, "peak_kind": f"{peaks['source']} copy",
+                           "frac_of_nominal": ach / NOMINAL_HBM_GBS, "nominal_peak": NOMINAL_HBM_GBS}
     dominant = max(roofs, key=lambda k: roofs[k]["ms_per_launch"]) if roofs else None
     attn_ms = sum(phase_ms.values()) / max(phase_calls["plan"], 1)
 
@@ -429,6 +433,7 @@ def main():
         "gpu_launches": int(launches),
         "attention_ms_per_step": attn_ms,
         "attention_tokens_per_s": world * tokens / (attn_ms * 1e-3) if attn_ms > 0 else None,
+        "ms_per_step_median": float(np.median(step_ms)), "ms_per_step_min": float(min(step_ms)),
         "ms_per_step_without_phase_events": plain_ms,
         "ms_per_step_cuda_graph": graph_ms,
         "phase_ms_per_step": {k: (phase_ms[k] / phase_calls[k] if phase_calls[k] else 0.0) for k in phase_ms},

@@ -55,6 +55,7 @@ struct Ctrl {
   // softmax warps its Q rows before item k has drained.
   int item_e[2];
   TileItem item[2];
+  alignas(16) int page_coord[2][32];             // row coordinates of the pages of four tiles, one block per producer warp
   int n_seg[2];                                  // page-segment tables of the chain, one copy per producer warp
   int seg_first_page[2][SS_MAX_DEPTH + 1];
   long long seg_page_off[2][SS_MAX_DEPTH];
@@ -136,6 +137,8 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
   uint32_t q_uses_tma = 0;  // ... of them chain items (their Q arrives through TMA and q_full_tma)
   uint32_t item_seq = 0;    // items this CTA has started
   int n_prefetched = 0;     // producer warps: tiles of the current item that were issued during the previous one
+  int prod_stage = 0;       // producer warps: ring stage of the next tile to issue, and how often the ring has wrapped
+  uint32_t prod_wraps = 0;  //   (kept as counters: a modulo by a stage count that differs per warp is a division per tile)
 
   // Takes the next item from the global counter into slot `dst` (one thread).
   auto fetch_item = [&](int dst) {
@@ -461,8 +464,8 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
       uint8_t* ring = smem + (which ? kOffV : kOffK);
       int* seg_first = C.seg_first_page[which];
       long long* seg_off = C.seg_page_off[which];
-      // tiles [j_begin, j_end) of item `v`, whose tile 0 has the global tile number g_base
-      auto stream_tiles = [&](const ItemView& v, uint32_t g_base, int j_begin, int j_end) -> bool {
+      // tiles [j_begin, j_end) of item `v`; calls follow one another in tile order, so the stage counters run on
+      auto stream_tiles = [&](const ItemView& v, int j_begin, int j_end) -> bool {
         if (j_begin >= j_end) return true;
         if (lane == 0) {
           int n_seg = 0;
@@ -505,35 +508,50 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
         };
         bool ok = true;
         // The page ids of four tiles are fetched with one load per lane (lane = 8 * tile-in-block + page), a whole
-        // block ahead of their use: the dependent global load is off the per-tile path.
+        // block ahead of their use: the dependent global load is off the per-tile path.  The lanes hand them to ONE
+        // elected lane through shared memory, and that lane issues all copies of the block in straight-line code:
+        // bulk-tensor copies are issued from uniform registers, and under a branch that several lanes may take the
+        // compiler wraps each of them in a loop over the active lanes (about a dozen instructions per copy, all of
+        // them issue slots taken from the softmax warp of the same sub-partition).
+        int* coords = C.page_coord[which];
         int cur = page_coord(j_begin + (lane >> 3), lane & 7);
         for (int j0 = j_begin; j0 < j_end && ok; j0 += 4) {
           const int nxt = page_coord(j0 + 4 + (lane >> 3), lane & 7);
-          for (int t = 0; t < 4 && j0 + t < j_end && ok; ++t) {
-            const int j = j0 + t;
-            const uint32_t gj = g_base + j;
-            const int s = gj % n_stages;
-            const uint32_t u = gj / n_stages;
-            const int pos0 = v.kv_begin + j * kTile;
-            const int n_pages = (min(kTile, v.kv_end - pos0) + kPage - 1) / kPage;
-            const int coord_y = __shfl_sync(0xffffffffu, cur, t * 8 + (lane & 7));
-            if (u > 0) ok = mbar_wait(&empty[s], (u - 1) & 1, abort_flag);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            if (lane == 0) mbar_arrive_expect_tx(&full[s], static_cast<uint32_t>(n_pages) * 4096u);
-            __syncwarp();
-            if (lane < n_pages) {
-              uint8_t* dst = ring + s * kStageBytes + lane * 2048;
-              tma_load_2d(dst, tm, 0, coord_y, &full[s]);
-              tma_load_2d(dst + kStageBytes / 2, tm, 64, coord_y, &full[s]);
+          const int n_blk = min(4, j_end - j0);
+          coords[lane] = cur;
+          __syncwarp();
+          if (elect_one()) {
+            int s = prod_stage;
+            uint32_t u = prod_wraps;
+            for (int t = 0; t < n_blk; ++t) {
+              const int pos0 = v.kv_begin + (j0 + t) * kTile;
+              const int n_pages = (min(kTile, v.kv_end - pos0) + kPage - 1) / kPage;
+              if (u > 0 && !mbar_wait(&empty[s], (u - 1) & 1, abort_flag)) { ok = false; break; }
+              mbar_arrive_expect_tx(&full[s], static_cast<uint32_t>(n_pages) * 4096u);
+              const int4 y03 = *reinterpret_cast<const int4*>(&coords[t * 8]);
+              const int4 y47 = *reinterpret_cast<const int4*>(&coords[t * 8 + 4]);
+              const int y[8] = {y03.x, y03.y, y03.z, y03.w, y47.x, y47.y, y47.z, y47.w};
+              uint8_t* dst = ring + s * kStageBytes;
+#pragma unroll
+              for (int pg = 0; pg < kTile / kPage; ++pg) {
+                if (pg < n_pages) {
+                  tma_load_2d(dst + pg * 2048, tm, 0, y[pg], &full[s]);
+                  tma_load_2d(dst + kStageBytes / 2 + pg * 2048, tm, 64, y[pg], &full[s]);
+                }
+              }
+              if (++s == n_stages) { s = 0; ++u; }
             }
           }
+          __syncwarp();                                          // the elected lane has read the coordinates
+          ok = __all_sync(0xffffffffu, ok);
+          prod_stage += n_blk;                                   // every lane keeps the counters
+          while (prod_stage >= n_stages) { prod_stage -= n_stages; ++prod_wraps; }
           cur = nxt;
         }
         __syncwarp();                                            // the segment tables are rewritten by the next call
         return ok;
       };
-      bool ok = stream_tiles(it, g_tile, n_prefetched, n_tiles);
+      bool ok = stream_tiles(it, n_prefetched, n_tiles);
       n_prefetched = 0;
       // ---- the first tiles of the next item --------------------------------------------------------------------
       if (ok) ok = mbar_wait(&C.item_ready[slot ^ 1], ((item_seq + 1) >> 1) & 1, abort_flag);
@@ -544,13 +562,13 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
           const ItemView nv = view(C.item[slot ^ 1]);
           n_prefetched = min(nv.n_tiles, n_stages);
           // Q buffer slot ^ 1 is free: the products of the item before this one have completed
-          if (which == 0 && lane == 0 && nv.n_tiles > 0 && nv.kind == kItemChain) q_tma_start(nv, slot ^ 1);
-          if (!stream_tiles(nv, g_tile + n_tiles, 0, n_prefetched)) n_prefetched = 0;   // (aborting)
+          if (which == 0 && nv.n_tiles > 0 && nv.kind == kItemChain && elect_one()) q_tma_start(nv, slot ^ 1);
+          if (!stream_tiles(nv, 0, n_prefetched)) n_prefetched = 0;   // (aborting)
         }
       }
     } else if (warp == kSoftmaxWarps + 2) {
       // =================================================== S = Q K^T issuer ====================================
-      if (lane == 0 && n_tiles > 0) {
+      if (n_tiles > 0 && elect_one()) {                          // (elected, not `lane == 0`: see the producers)
         constexpr uint32_t idesc_qk = instr_desc_bf16(128, kTile, false);
         const uint64_t q_desc0 = smem_desc_sw128(smem_u32(smem + kOffQ + slot * 32768), 0, 1024);
         const uint64_t k_desc0 = smem_desc_sw128(smem_u32(smem + kOffK), 0, 1024);
@@ -577,7 +595,7 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
       }
     } else {
       // =================================================== O += P V issuer =====================================
-      if (lane == 0 && n_tiles > 0) {
+      if (n_tiles > 0 && elect_one()) {
         constexpr uint32_t idesc_pv = instr_desc_bf16(128, kHeadDim, true);
         const uint64_t v_desc0 = smem_desc_sw128(smem_u32(smem + kOffV), kStageBytes / 2, 1024);
         bool ok = true;

@@ -47,17 +47,35 @@ __device__ __forceinline__ bool mbar_try_wait_suspend(uint64_t* bar, uint32_t pa
   return ok != 0;
 }
 // Bounded wait.  `abort_flag` lives in shared memory and is raised by whoever gives up first.
+// A waiting thread shares its sub-partition's issue slots with a softmax warp, so the retry loop is kept to the test
+// and a counter; the abort flag and the clock are looked at on every 16th retry only (each retry is itself bounded
+// by the hardware's suspend limit).
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
   if (mbar_try_wait(bar, parity)) return true;
-  const long long t0 = clock64();
+  long long t0 = 0;
+  uint32_t spins = 0;
   while (!mbar_try_wait_suspend(bar, parity, 20000u)) {
+    if ((++spins & 15u) != 0u) continue;
     if (*abort_flag) return false;
-    if (clock64() - t0 > kWaitCycles) {
+    if (t0 == 0) {
+      t0 = clock64();
+    } else if (clock64() - t0 > kWaitCycles) {
       *abort_flag = 1;
       return false;
     }
   }
   return true;
+}
+// Whole (converged) warp: true in exactly one lane.  Code guarded by it is known to the compiler to run in a single
+// thread, so tcgen05 / bulk-tensor instructions inside take their uniform-register operands directly.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred = 0;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "elect.sync _|p, 0xffffffff;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(pred)::"memory");
+  return pred != 0;
 }
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 // Makes generic-proxy writes to shared memory visible to the async proxy (TMA, tcgen05.mma operand reads).
