@@ -411,6 +411,7 @@ def main():
                           "unit": "TFLOP/s", "frac": ach / tensor_peak, "traffic": traffic.get("tiles"),
                           "ms_per_launch": t_ms, "peak_kind": f"{peaks['source']} {'sustained' if long_step else 'burst'}",
                           "frac_of_nominal": ach / NOMINAL_BF16_TFLOPS, "nominal_peak": NOMINAL_BF16_TFLOPS,
+                          "frac_of_sustained": ach / peaks["bf16_sustained"],
                           "ctas_per_sm": 2 if args.tiles_2cta else 1}
     if phase_calls["leaves"]:
         t_ms = phase_ms["leaves"] / phase_calls["leaves"]

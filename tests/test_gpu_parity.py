@@ -304,6 +304,32 @@ def test_attention_shapes(shape, mode, flags):
     check_attention(r, w, ref, max_paths=64)
 
 
+@pytest.mark.parametrize("seed", range(8))
+def test_attention_random_trees(seed):
+    """Seeded random tree shapes (depth, fan-out, head grouping, leaf and step lengths, duplicates) through the
+    default kernels: item boundaries, ragged tiles, page tails and empty leaves fall differently in each."""
+    rng = np.random.default_rng(9000 + seed)
+    Hkv = int(rng.choice([1, 2, 4, 8]))
+    G = int(rng.choice([1, 2, 4, 6, 7, 8, 16]))
+    depth = int(rng.integers(1, 4))
+    levels = [int(rng.choice([0, 16, 40, 128, 300, 700])) for _ in range(depth)]
+    fanout = [int(rng.integers(1, 6)) for _ in range(depth - 1)] + [int(rng.integers(2, 40))]
+    leaf = (int(rng.integers(0, 3)), int(rng.choice([20, 130, 400])))
+    style = int(rng.integers(0, 3))
+
+    def qfn(i, n, r):
+        if style == 0:
+            return 1
+        if style == 1:
+            return int(r.integers(1, 140))
+        return 1 if i % 2 else int(r.integers(16, 129))
+
+    w = synth.build_tree_workload(f"fuzz{seed}", 77000 + seed, Hkv * G, Hkv, levels, fanout, int(rng.integers(1, 4)), leaf, qfn,
+                                  dup_frac=float(rng.choice([0.0, 0.2])))
+    r, ref = attention_only(w, 0)
+    check_attention(r, w, ref, max_paths=48)
+
+
 @pytest.mark.parametrize("mode,flags", MODES)
 def test_attention_closed_forms(mode, flags):
     """Q == 0 => lse = ln(visible), out = mean of the visible V rows; with V[j,:] = position j (< 256, exact in
