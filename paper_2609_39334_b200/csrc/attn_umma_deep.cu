@@ -12,8 +12,10 @@
 // Roles: warps 0-3 softmax + epilogue (one query row per thread = one TMEM lane); warp 4 streams K tiles and warp 5
 // V tiles through TMA (3 and 2 stages of 32 KB); warp 6 lane 0 issues S[b] = Q K^T (8 MMAs per tile), warp 7 lane 0
 // issues O += P[b] V (8 MMAs, P read from TMEM where it overwrote the first 64 columns of S[b], V MN-major), lane 1
-// of warp 7 fetches the NEXT item while this one runs: the producers then load its first K / V tiles and the softmax
-// warps copy its Q rows (cp.async into the second Q buffer) before the current item has drained.
+// of warp 7 fetches the NEXT item while this one runs: the producers then load its first K / V tiles and its Q rows
+// (a 3-D TMA box for a chain item, issued by the K producer; cp.async of the gathered rows of a stacked item by the
+// V producer warp) into the second Q buffer before the current item has drained.  The softmax warps do nothing but
+// the softmax and the epilogue: every other duty that sat in their loop cost more than it looked.
 // Every wait is bounded; on expiry the CTA raises its abort flag, all roles fall through to the item-end barrier,
 // the CTA frees its TMEM and the kernel records SS_ERR_TIMEOUT.
 #include "attn_plan.cuh"
@@ -104,7 +106,7 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
 
   if (tid == 0) {
     C.abort_flag = (smem_u32(smem) & 1023u) ? 1 : 0;
-    mbar_init(&C.q_full, kSoftmaxWarps * 32);       // stacked items: the softmax threads copy the (gathered) rows
+    mbar_init(&C.q_full, 1);                        // stacked items: the V producer warp copies the (gathered) rows
     mbar_init(&C.q_full_tma, 1);                    // chain items: one TMA box pair
     for (int s = 0; s < kStagesK; ++s) { mbar_init(&C.k_full[s], 1); mbar_init(&C.k_empty[s], 1); }
     for (int s = 0; s < kStagesV; ++s) { mbar_init(&C.v_full[s], 1); mbar_init(&C.v_empty[s], 1); }
@@ -149,21 +151,25 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
     __threadfence_block();
     mbar_arrive(&C.item_ready[dst]);
   };
-  // Softmax threads: start the asynchronous copy of item `v`'s Q rows into Q buffer `buf` (UMMA K-major layout with
-  // the 128-byte swizzle; rows past the item's last one are zero-filled).  Completed by q_copy_wait().
-  auto q_copy_start = [&](const ItemView& v, int buf) {
-    const int row = tid;
-    const int i = row / G, hl = row - i * G;
-    const bool row_valid = i < v.n_tok;
-    int64_t q_src = 0;
-    if (row_valid) q_src = (v.kind == kItemChain) ? static_cast<int64_t>(v.src0 + i) : P.dec_src[v.tok0 + i];
-    const char* src = reinterpret_cast<const char*>(P.q + (q_src * P.Hq + (v.g * G + hl)) * kHeadDim);
+  // Stacked items: one producer warp starts the asynchronous copy of item `v`'s (gathered) Q rows into Q buffer `buf`
+  // (UMMA K-major layout with the 128-byte swizzle; rows past the item's last one are zero-filled).  The softmax
+  // warps used to do this inside their tile loop, where the dependent load of the row index and the hundred
+  // instructions of the copy cost each of them about 1400 clocks per item.
+  auto q_gather_start = [&](const ItemView& v, int buf) {
     const uint32_t dst0 = smem_u32(smem + kOffQ + buf * 32768);
-    const uint32_t n_src = row_valid ? 16u : 0u;                 // 0 source bytes: the 16 destination bytes are zeroed
+#pragma unroll 1
+    for (int row = lane; row < 128; row += 32) {
+      const int i = row / G, hl = row - i * G;
+      const bool row_valid = i < v.n_tok;
+      int64_t q_src = 0;
+      if (row_valid) q_src = P.dec_src[v.tok0 + i];
+      const char* src = reinterpret_cast<const char*>(P.q + (q_src * P.Hq + (v.g * G + hl)) * kHeadDim);
+      const uint32_t n_src = row_valid ? 16u : 0u;               // 0 source bytes: the 16 destination bytes are zeroed
 #pragma unroll
-    for (int ch = 0; ch < 16; ++ch)
-      asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst0 + (ch >> 3) * 16384 + sw128_offset(row, ch & 7)),
-                   "l"(src + ch * 16), "r"(n_src) : "memory");
+      for (int ch = 0; ch < 16; ++ch)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst0 + (ch >> 3) * 16384 + sw128_offset(row, ch & 7)),
+                     "l"(src + ch * 16), "r"(n_src) : "memory");
+    }
     asm volatile("cp.async.commit_group;" ::: "memory");
   };
 
@@ -179,12 +185,13 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
 
   if (tid == 0) fetch_item(0);
   __syncthreads();
-  if (warp < kSoftmaxWarps) {                                    // Q of the first item
-    if (mbar_wait(&C.item_ready[0], 0, abort_flag)) {
+  bool q_pending = false;   // V producer warp: a gather of the coming item's Q rows is under way
+  if (warp == kSoftmaxWarps + 1) {                               // Q of a first stacked item
+    if (__all_sync(0xffffffffu, mbar_wait(&C.item_ready[0], 0, abort_flag))) {
       const int e0 = C.item_e[0];
       if (e0 >= 0 && e0 < n_items) {
         const ItemView v0 = view(C.item[0]);
-        if (v0.n_tiles > 0 && v0.kind != kItemChain) q_copy_start(v0, 0);
+        if (v0.n_tiles > 0 && v0.kind != kItemChain) { q_gather_start(v0, 0); q_pending = true; }
       }
     }
   }
@@ -214,33 +221,16 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
       const int i = row / G, hl = row - i * G;
       const bool row_valid = i < it.n_tok;
       const int h = it.g * G + hl;
-      int64_t q_row = 0, q_src = 0;                               // output row / row of q holding the query
+      int64_t q_row = 0;                                          // output row
       int dec = 0;
       if (row_valid) {
-        if (it.kind == kItemChain) { q_row = it.tok0 + i; q_src = it.src0 + i; }
-        else { dec = it.tok0 + i; q_row = P.dec_tok[dec]; q_src = P.dec_src[dec]; }
+        if (it.kind == kItemChain) q_row = it.tok0 + i;
+        else { dec = it.tok0 + i; q_row = P.dec_tok[dec]; }
       }
       const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
       float m = -INFINITY, m_next = -INFINITY, l = 0.f;
       bool ok = true;
-      // Q rows of the next item -> the other Q buffer (free: the products of item k-1 have completed), once the
-      // descriptor of that item has been published; called after the first tile so that the wait is over already.
-      auto start_next_q = [&]() {
-        if (!mbar_wait(&C.item_ready[slot ^ 1], ((item_seq + 1) >> 1) & 1, abort_flag)) return;
-        const int e_next = C.item_e[slot ^ 1];
-        if (e_next < 0 || e_next >= n_items) return;
-        const ItemView nv = view(C.item[slot ^ 1]);
-        if (nv.n_tiles > 0 && nv.kind != kItemChain) q_copy_start(nv, slot ^ 1);
-      };
-      if (n_tiles == 0) start_next_q();
       if (n_tiles > 0) {
-        // ---- Q rows of a stacked item: their asynchronous copy was started during the previous item (a chain item's
-        //      rows come through TMA, issued by the K producer) --------------------------------------------------------
-        if (it.kind != kItemChain) {
-          asm volatile("cp.async.wait_group 0;" ::: "memory");
-          fence_proxy_async_smem();
-          mbar_arrive(&C.q_full);
-        }
         int limit_row = (it.kind == kItemChain) ? it.limit0 + i : it.limit0;
         if (limit_row > it.kv_end) limit_row = it.kv_end;
         // first tile in which some row of this warp has a masked column (causal tail / end of the source): tiles
@@ -398,7 +388,6 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
           if (n_keys < kTile) fence_proxy_async_smem();           // the V rows cleared above
           tc_fence_before();
           mbar_arrive(&C.p_full[b]);
-          if (j == (n_tiles > 1 ? 1 : 0)) start_next_q();
         }
         if (ok) {
           ok = mbar_wait(&C.o_final, q_uses & 1, abort_flag);
@@ -551,6 +540,13 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
         __syncwarp();                                            // the segment tables are rewritten by the next call
         return ok;
       };
+      if (which == 1 && q_pending) {                               // the Q rows gathered during the previous item
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&C.q_full);
+        q_pending = false;
+      }
       bool ok = stream_tiles(it, n_prefetched, n_tiles);
       n_prefetched = 0;
       // ---- the first tiles of the next item --------------------------------------------------------------------
@@ -563,6 +559,8 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
           n_prefetched = min(nv.n_tiles, n_stages);
           // Q buffer slot ^ 1 is free: the products of the item before this one have completed
           if (which == 0 && nv.n_tiles > 0 && nv.kind == kItemChain && elect_one()) q_tma_start(nv, slot ^ 1);
+          // Q buffer slot ^ 1 is free: the products of the item before this one have completed
+          if (which == 1 && nv.n_tiles > 0 && nv.kind != kItemChain) { q_gather_start(nv, slot ^ 1); q_pending = true; }
           if (!stream_tiles(nv, 0, n_prefetched)) n_prefetched = 0;   // (aborting)
         }
       }
