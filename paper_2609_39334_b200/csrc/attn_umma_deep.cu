@@ -81,6 +81,14 @@ __device__ __forceinline__ uint32_t pack_bf16_rn(float a, float b) {
   return *reinterpret_cast<uint32_t*>(&pk);
 }
 
+// 32-byte store (a whole sector per lane: the epilogue writes one row per thread, so a 16-byte store leaves half of
+// every sector for a second transaction).  `p` must be 32-byte aligned.
+__device__ __forceinline__ void st_global_32B(void* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d, uint32_t e, uint32_t f,
+                                              uint32_t g, uint32_t h) {
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(a), "r"(b), "r"(c), "r"(d), "r"(e),
+               "r"(f), "r"(g), "r"(h) : "memory");
+}
+
 struct ItemView {
   int node, tok0, n_tok, kind, g, kv_begin, kv_end, limit0, slot_off, src0, n_tiles;
 };
@@ -414,24 +422,24 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
           }
           if (!row_valid) continue;
           if (final_out) {
-            uint4* dst = reinterpret_cast<uint4*>(P.out + (q_row * P.Hq + h) * kHeadDim + c0);
+            __nv_bfloat16* dst = P.out + (q_row * P.Hq + h) * kHeadDim + c0;
 #pragma unroll
-            for (int x = 0; x < 4; ++x) {
-              uint32_t w[4];
+            for (int x = 0; x < 2; ++x) {
+              uint32_t w[8];
 #pragma unroll
-              for (int y = 0; y < 4; ++y) {
-                __nv_bfloat162 pk = __floats2bfloat162_rn(__uint_as_float(orow[8 * x + 2 * y]) * inv,
-                                                          __uint_as_float(orow[8 * x + 2 * y + 1]) * inv);
-                w[y] = *reinterpret_cast<uint32_t*>(&pk);
-              }
-              dst[x] = make_uint4(w[0], w[1], w[2], w[3]);
+              for (int y = 0; y < 8; ++y)
+                w[y] = pack_bf16_rn(__uint_as_float(orow[16 * x + 2 * y]) * inv, __uint_as_float(orow[16 * x + 2 * y + 1]) * inv);
+              st_global_32B(dst + 16 * x, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]);
             }
           } else {
-            float4* dst = reinterpret_cast<float4*>(P.part_o + (slot * P.Hq + h) * kHeadDim + c0);
+            float* dst = P.part_o + (slot * P.Hq + h) * kHeadDim + c0;
 #pragma unroll
-            for (int x = 0; x < 8; ++x)
-              dst[x] = make_float4(__uint_as_float(orow[4 * x]) * inv, __uint_as_float(orow[4 * x + 1]) * inv,
-                                   __uint_as_float(orow[4 * x + 2]) * inv, __uint_as_float(orow[4 * x + 3]) * inv);
+            for (int x = 0; x < 4; ++x) {
+              uint32_t w[8];
+#pragma unroll
+              for (int y = 0; y < 8; ++y) w[y] = __float_as_uint(__uint_as_float(orow[8 * x + y]) * inv);
+              st_global_32B(dst + 8 * x, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]);
+            }
           }
         }
         if (row_valid) {
