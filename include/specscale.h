@@ -448,6 +448,13 @@ int32_t ss_debug_tile_kernel_occupancy(void);
 int32_t ss_debug_umma_tile(const void* a_bf16, const void* b_bf16, float* c, int32_t n, int32_t k,
                            int32_t b_is_mn_major, int32_t* status_out, void* stream);
 
+/* Self-test of the bounded wait every kernel role uses (no paper counterpart): one CTA waits on a shared-memory
+ * barrier that nothing ever completes.  The wait must give up after its time limit (about 0.2 s), raise the CTA's
+ * abort flag and return, and the kernel must then end normally.  status_out: device int32[2];
+ * status_out[0] receives SS_ERR_TIMEOUT when that happened (SS_OK if the wait claimed success, which would be a bug),
+ * status_out[1] the clocks the wait took, in millions.  Returns SS_OK when the kernel was launched. */
+int32_t ss_debug_bounded_wait(int32_t* status_out, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

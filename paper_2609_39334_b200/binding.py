@@ -33,7 +33,7 @@ SS_DEDUP_STATIC_MAX_PATHS = 65536
 EXPORTS = [
     "ss_status_string", "ss_last_device_status", "ss_dedup_workspace_bytes", "ss_dedup_paths",
     "ss_tree_attention_workspace_bytes", "ss_tree_attention", "ss_topk_workspace_bytes", "ss_topk_prune",
-    "ss_launch_count", "ss_debug_umma_tile", "ss_profile_enable", "ss_profile_read",
+    "ss_launch_count", "ss_debug_umma_tile", "ss_debug_bounded_wait", "ss_profile_enable", "ss_profile_read",
     "ss_dedup_paths_static", "ss_debug_tile_kernel_occupancy", "ss_early_prune",
     "ss_branch_sample", "ss_gather_unique_paths", "ss_candidate_step_host_arena_bytes", "ss_candidate_step_host",
     "ss_prefix_tree_workspace_bytes", "ss_build_prefix_tree",
@@ -345,6 +345,10 @@ def ss_branch_sample(logits, draw_offsets, uniforms, n_seq, vocab, temperature, 
     if check:
         _check(rc, "ss_branch_sample")
     return rc
+
+
+def ss_debug_bounded_wait(status_out, stream=None) -> int:
+    return lib().ss_debug_bounded_wait(_ptr(status_out), _stream(stream))
 
 
 def ss_debug_umma_tile(a, b, c, n, k, b_is_mn_major, status_out, stream=None) -> int:

@@ -128,8 +128,38 @@ __global__ void __launch_bounds__(128) umma_tile_test_kernel(const __grid_consta
   if (tid == 0) *status = abort_flag ? SS_ERR_TIMEOUT : SS_OK;
 }
 
+// The bounded wait on a barrier that nothing completes: must return false after its limit, with the abort flag set.
+__global__ void __launch_bounds__(64) bounded_wait_test_kernel(int32_t* status) {
+  ss::grid_dependency_enter();
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(&bar, 1);
+    fence_barrier_init();
+  }
+  __syncthreads();
+  const long long t0 = clock64();
+  // thread 0 runs into the limit itself; thread 32 is released by the flag thread 0 raises (or by its own limit)
+  bool gave_up = true;
+  if (threadIdx.x == 0 || threadIdx.x == 32) gave_up = !mbar_wait(&bar, 0, &abort_flag);
+  const long long dt = clock64() - t0;
+  const int all_gave_up = __syncthreads_and(gave_up ? 1 : 0);
+  if (threadIdx.x == 0) {
+    status[0] = (all_gave_up && abort_flag != 0) ? SS_ERR_TIMEOUT : SS_OK;
+    status[1] = static_cast<int32_t>(dt / 1000000);
+  }
+}
+
 }  // namespace umma
 }  // namespace ss
+
+extern "C" int32_t ss_debug_bounded_wait(int32_t* status_out, void* stream) {
+  using namespace ss;
+  if (!status_out) return SS_ERR_INVALID_ARG;
+  SS_LAUNCH(umma::bounded_wait_test_kernel, 1, 64, 0, as_stream(stream), status_out);
+  return SS_OK;
+}
 
 extern "C" int32_t ss_debug_umma_tile(const void* a_bf16, const void* b_bf16, float* c, int32_t n, int32_t k,
                                       int32_t b_is_mn_major, int32_t* status_out, void* stream) {

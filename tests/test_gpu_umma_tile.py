@@ -26,3 +26,18 @@ def test_umma_tile_product(n, k, b_mn):
     # fp32 accumulation of exact bf16 products: error ~ k * 2^-24 * |terms|
     assert torch.isfinite(got).all()
     assert (got - want).abs().max().item() < 1e-3 * (k / 64) ** 0.5 + 1e-4
+
+
+@pytest.mark.gpu
+def test_bounded_wait_gives_up_and_the_kernel_ends():
+    """Every role of the tensor-core kernels waits through one bounded helper; on a barrier that nothing completes it
+    must return after its limit with the CTA's abort flag raised, and the context must stay usable."""
+    dev = torch.device("cuda:0")
+    status = torch.full((2,), -1, dtype=torch.int32, device=dev)
+    assert B.ss_debug_bounded_wait(status) == B.SS_OK
+    torch.cuda.synchronize()
+    st = status.cpu().tolist()
+    assert st[0] == B.SS_ERR_TIMEOUT
+    assert 100 <= st[1] <= 4000          # ~0.2 s worth of clocks, in millions
+    x = torch.arange(8, device=dev).sum().item()      # the context still works
+    assert x == 28
