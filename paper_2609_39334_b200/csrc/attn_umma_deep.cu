@@ -248,9 +248,9 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
           const uint32_t gj = g_tile + j;
           const int b = gj % kRing;
           const uint32_t s_col = kColS + b * kTile;
-          ok = mbar_wait(&C.s_full[b], (gj / kRing) & 1, abort_flag);
-          ok = __all_sync(0xffffffffu, ok);
-          if (!ok) break;
+          // (no vote and no early exit here: after a wait has run out the CTA is aborting, the later waits fail fast
+          // and the thread runs the rest of the item on whatever it finds; `ok` keeps the result from being written)
+          if (!mbar_wait(&C.s_full[b], (gj / kRing) & 1, abort_flag)) ok = false;
           tc_fence_after();
           // the second half of the scores is fetched while the exponentials of the first half are computed
           uint32_t sr[kTile];
@@ -397,6 +397,7 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
           tc_fence_before();
           mbar_arrive(&C.p_full[b]);
         }
+        ok = __all_sync(0xffffffffu, ok);
         if (ok) {
           ok = mbar_wait(&C.o_final, q_uses & 1, abort_flag);
           ok = __all_sync(0xffffffffu, ok);
