@@ -15,6 +15,9 @@ LIB = os.path.join(_HERE, "libspecscale.so")
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "--expt-relaxed-constexpr",
          "-Xcompiler", "-fPIC"]
+# Per-file additions.  The softmax threads of the default tile kernel sit at the 254-register limit; ptxas's most
+# register-conserving setting schedules their loop slightly better (measured: +0.8 % on the tile kernel).
+FILE_FLAGS = {"attn_umma_deep.cu": ["-Xptxas", "--register-usage-level=10"]}
 
 
 def sources():
@@ -40,7 +43,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     for src in sources():
         obj = os.path.join(objdir, os.path.basename(src)[:-3] + ".o")
         objs.append(obj)
-        cmd = [NVCC, *FLAGS, "-c", src, "-o", obj]
+        cmd = [NVCC, *FLAGS, *FILE_FLAGS.get(os.path.basename(src), []), "-c", src, "-o", obj]
         if verbose:
             cmd.insert(1, "-Xptxas")
             cmd.insert(2, "-v")
