@@ -406,7 +406,7 @@ def main():
     if phase_calls["tiles"]:
         t_ms = phase_ms["tiles"] / phase_calls["tiles"]
         ach = work["tile_flops"] / (t_ms * 1e-3) / 1e12
-        roofs["tiles"] = {"kernel": "tile_items_umma_kernel" if args.tiles_2cta else "tile_items_umma_deep_kernel",
+        roofs["tiles"] = {"kernel": "tile_items_umma_kernel" if args.tiles_2cta else "tile_items_umma_split_kernel",
                           "bound": "tensor", "achieved": ach, "peak": tensor_peak,
                           "unit": "TFLOP/s", "frac": ach / tensor_peak, "traffic": traffic.get("tiles"),
                           "ms_per_launch": t_ms, "peak_kind": f"{peaks['source']} {'sustained' if long_step else 'burst'}",

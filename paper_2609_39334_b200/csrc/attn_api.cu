@@ -15,7 +15,7 @@ int32_t launch_leaf_items_simple(const Params& P, cudaStream_t st, int sm_count)
 int32_t launch_merge(const Params& P, cudaStream_t st, int sm_count);
 int32_t launch_leaf_items(const Params& P, cudaStream_t st, int sm_count);
 int32_t launch_tile_items_umma(const Params& P, cudaStream_t st, int sm_count);
-int32_t launch_tile_items_umma_deep(const Params& P, cudaStream_t st, int sm_count);
+int32_t launch_tile_items_umma_split(const Params& P, cudaStream_t st, int sm_count);
 
 // ---- per-phase event timing (diagnostics) ------------------------------------------------------------------
 constexpr int kProfCalls = 256;                      // timed calls between two reads
@@ -212,7 +212,7 @@ extern "C" int32_t ss_tree_attention(const ss_attn_desc_t* d, void* workspace, s
   if (rc == SS_OK && any && !generic_only) {
     const bool two_cta = (d->flags & SS_FLAG_TILES_2CTA) != 0;
     rc = simple ? launch_tile_items_simple(P, st, sms)
-                : (two_cta ? launch_tile_items_umma(P, st, sms) : launch_tile_items_umma_deep(P, st, sms));
+                : (two_cta ? launch_tile_items_umma(P, st, sms) : launch_tile_items_umma_split(P, st, sms));
     ran(SS_PHASE_TILES);
   }
   mark(SS_PHASE_LEAVES);

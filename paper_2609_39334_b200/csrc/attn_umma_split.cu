@@ -1,24 +1,37 @@
-// Tensor-core tile kernel of ss_tree_attention, deep-pipeline version (tcgen05 + TMEM + TMA): one CTA per SM that owns
-// all 512 TMEM columns and works on 128-key tiles.  Same items and the same arithmetic as the two-CTAs-per-SM kernel in
-// attn_umma.cu (a 64-key tile there); what differs follows from three measurements on this part:
+// Tensor-core tile kernel of ss_tree_attention (tcgen05 + TMEM + TMA), the default: one CTA per SM that owns all 512
+// TMEM columns and works on 128-key tiles.  Same items and the same arithmetic as the two-CTAs-per-SM kernel in
+// attn_umma.cu (a 64-key tile there); what differs follows from measurements on this part:
 //   * an SM retires one tcgen05 instruction (MMA or commit) per ~50 clocks whatever its shape, and a 64-key tile costs
 //     17 of them: with 128-key tiles every MMA is M128 x N128 x K16 (64 clocks of math) and the count per key halves;
-//   * an ex2 holds an SM sub-partition for 8 clocks and every other instruction of the softmax loop ADDS to that (the
-//     pipes do not overlap in issue), so the loop works on packed fp32 pairs, takes the row maximum from a sample of
-//     the columns inside the exponential loop, and uses a reference maximum that lags one tile behind;
+//   * an ex2 holds an SM sub-partition for 8 clocks and every other instruction issued there ADDS to that (the pipes
+//     do not overlap in issue), so the loop works on packed fp32 pairs, takes the row maximum from a sample of the
+//     columns inside the exponential loop, and uses a reference maximum that lags one tile behind;
 //   * a score buffer is recycled only when the P V product that read it has completed, so with two buffers the chain
 //     Q K^T -> softmax -> P V of one tile bounds the next but one: three S/P buffers (128 columns each) + O (128
-//     columns) fill the TMEM exactly, Q stays in shared memory.
-// Roles: warps 0-3 softmax + epilogue (one query row per thread = one TMEM lane); warp 4 streams K tiles and warp 5
-// V tiles through TMA (3 and 2 stages of 32 KB); warp 6 lane 0 issues S[b] = Q K^T (8 MMAs per tile), warp 7 lane 0
-// issues O += P[b] V (8 MMAs, P read from TMEM where it overwrote the first 64 columns of S[b], V MN-major), lane 1
-// of warp 7 fetches the NEXT item while this one runs: the producers then load its first K / V tiles and its Q rows
-// (a 3-D TMA box for a chain item, issued by the K producer; cp.async of the gathered rows of a stacked item by the
-// V producer warp) into the second Q buffer before the current item has drained.  The softmax warps do nothing but
-// the softmax and the epilogue: every other duty that sat in their loop cost more than it looked.
-// Every wait is bounded; on expiry the CTA raises its abort flag, all roles fall through to the item-end barrier,
-// the CTA frees its TMEM and the kernel records SS_ERR_TIMEOUT.
+//     columns) fill the TMEM exactly, Q stays in shared memory;
+//   * with one softmax thread per row that thread needs all 254 registers and spends a third of each tile in exposed
+//     latencies.  Here TWO threads share a row: the two warps that can reach a TMEM lane quarter (w and w + 4) each
+//     take 64 of the row's 128 scores, so a thread holds 64 scores + 32 packed P values (168 registers are plenty)
+//     and each sub-partition has two softmax warps to interleave.
+// What the two threads of a row must agree on is the reference maximum.  For the first tile of an item they exchange
+// the exact maxima of their halves (a 64-thread barrier, once per item); from then on each posts the sampled maximum
+// of its half to a shared-memory mailbox after every tile and reads the other's post of the PREVIOUS tile, so both
+// compute the same lagged reference without waiting for each other.  P of the two halves goes over the first 32
+// columns of each thread's own 64 score columns (columns 0..31 and 64..95 of the S buffer).  Row sums are kept per
+// half and added in the epilogue (second 64-thread barrier), where each half also writes 64 output columns.  A half
+// row whose exponentials leave the range of the lagged reference (scores rising by more than 2^40 from one tile to
+// the next) cannot be repaired in place, because the other half has used the same reference: it marks the item, and
+// when the item's tiles are through, all warps of the CTA recompute it exactly on the CUDA cores (attn_rows.cuh).
+// Roles: warps 0-7 softmax + epilogue; warp 8 streams K tiles and warp 9 V tiles through TMA (3 and 2 stages of
+// 32 KB); an elected lane of warp 10 issues S[b] = Q K^T (8 MMAs per tile), of warp 11 O += P[b] V (8 MMAs, P read
+// from TMEM, V MN-major); lane 1 of warp 11 fetches the NEXT item while this one runs: the producers then load its
+// first K / V tiles and its Q rows (a 3-D TMA box for a chain item, issued by the K producer; cp.async of the
+// gathered rows of a stacked item by the V producer warp) into the second Q buffer before the current item has
+// drained.  The softmax warps do nothing but the softmax and the epilogue.
+// Every wait is bounded; on expiry the CTA raises its abort flag, the later waits fail fast, the roles run through
+// the item's remaining tiles without writing results, the CTA frees its TMEM and the kernel records SS_ERR_TIMEOUT.
 #include "attn_plan.cuh"
+#include "attn_rows.cuh"
 #include "umma.cuh"
 
 namespace ss {
@@ -26,9 +39,9 @@ namespace attn {
 
 using namespace umma;
 
-namespace deep {
+namespace split {
 
-constexpr int kSoftmaxWarps = 4;
+constexpr int kSoftmaxWarps = 8;               // two warps per TMEM lane quarter: each takes 64 of a row's 128 scores
 constexpr int kUmmaThreads = (kSoftmaxWarps + 4) * 32;
 constexpr int kTile = 128;                     // keys per tile (two of the planner's 64-key tiles)
 constexpr int kStageBytes = kTile * 256;       // one K or V tile: [2 halves of 64 dims][kTile rows][128 B]
@@ -58,6 +71,13 @@ struct Ctrl {
   int item_e[2];
   TileItem item[2];
   alignas(16) int page_coord[2][32];             // row coordinates of the pages of four tiles, one block per producer warp
+  // Sampled tile maxima of the two halves of a row, one tile behind: [tile parity][half][row], the low two bits of the
+  // value replaced by a tag (1 or 2) that tells the reader which tile the value belongs to.  The two exchanges per
+  // item that go through a pair barrier (exact maximum of the first tile, row sums at the end) borrow the slot that
+  // is idle at that moment and leave it cleared (tag 0 matches nothing).
+  uint32_t xmax[2][2][128];
+  int overflow[2];                               // (per item slot) a half-row left the range of the lagged reference:
+                                                 // the item is computed again, exactly, when its tiles are through
   int n_seg[2];                                  // page-segment tables of the chain, one copy per producer warp
   int seg_first_page[2][SS_MAX_DEPTH + 1];
   long long seg_page_off[2][SS_MAX_DEPTH];
@@ -89,6 +109,15 @@ __device__ __forceinline__ void st_global_32B(void* p, uint32_t a, uint32_t b, u
                "r"(f), "r"(g), "r"(h) : "memory");
 }
 
+__device__ __forceinline__ uint32_t ld_shared_volatile(uint32_t addr) {
+  uint32_t v;
+  asm volatile("ld.volatile.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_shared(uint32_t addr, uint32_t v) {
+  asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+
 struct ItemView {
   int node, tok0, n_tok, kind, g, kv_begin, kv_end, limit0, slot_off, src0, n_tiles;
 };
@@ -103,9 +132,15 @@ __device__ __forceinline__ ItemView view(const TileItem& it) {
   return v;
 }
 
+// Out of line on purpose: code that is inlined into the kernel costs its hot loops registers and instruction-cache
+// space even when it never runs.
+__device__ __noinline__ void exact_second_pass(const Params& P, const TileItem* it, int warp, int lane) {
+  tile_item_rows_exact(P, *it, warp, kUmmaThreads / 32, lane);
+}
+
 __global__ void __launch_bounds__(kUmmaThreads, 1)
-tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
-                            const __grid_constant__ CUtensorMap tmap_q, const Params P) {
+tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
+                            const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ Params P) {
   ss::grid_dependency_enter();
   extern __shared__ __align__(1024) uint8_t smem[];
   __shared__ Ctrl C;
@@ -130,6 +165,8 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
     prefetch_tensormap(&tmap_q);
   }
   for (int x = tid; x < 65536 / 16; x += kUmmaThreads) reinterpret_cast<uint4*>(smem + kOffQ)[x] = make_uint4(0, 0, 0, 0);
+  for (int x = tid; x < 2 * 2 * 128; x += kUmmaThreads) (&C.xmax[0][0][0])[x] = 0u;   // tag 0: nothing posted
+  if (tid == 0) C.overflow[0] = C.overflow[1] = 0;
   fence_proxy_async_smem();
   if (warp == kSoftmaxWarps) tmem_alloc(&C.tmem_slot, kTmemCols);
   tc_fence_before();
@@ -224,8 +261,12 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
 
     if (warp < kSoftmaxWarps) {
       // =================================================== softmax + epilogue ==================================
-      // One thread per query row (= one TMEM lane), 128 score columns per tile.
-      const int row = tid;
+      // Two threads per query row (= TMEM lane): thread `hf` of the pair takes score columns [64 hf, 64 hf + 64) of
+      // every tile, keeps its own partial row sum and writes output columns [64 hf, 64 hf + 64).  Both derive the
+      // same reference maximum: from the exact half maxima of the first tile (exchanged through a pair barrier) and,
+      // one tile behind, from the sampled maxima that each posts for the other.
+      const int hf = warp >> 2;
+      const int row = tid & 127;
       const int i = row / G, hl = row - i * G;
       const bool row_valid = i < it.n_tok;
       const int h = it.g * G + hl;
@@ -235,83 +276,92 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
         if (it.kind == kItemChain) q_row = it.tok0 + i;
         else { dec = it.tok0 + i; q_row = P.dec_tok[dec]; }
       }
-      const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
-      float m = -INFINITY, m_next = -INFINITY, l = 0.f;
+      const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
+      auto pair_barrier = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(2 + (warp & 3)) : "memory"); };
+      float m = 0.f, l = 0.f;                                     // reference maximum (0 while the row has no visible key)
+      uint32_t own_post = 0;                                      // what this thread posted for the previous tile
       bool ok = true;
       if (n_tiles > 0) {
         int limit_row = (it.kind == kItemChain) ? it.limit0 + i : it.limit0;
         if (limit_row > it.kv_end) limit_row = it.kv_end;
-        // first tile in which some row of this warp has a masked column (causal tail / end of the source): tiles
-        // before it need neither the mask nor a vote about it
         const int first_masked_tile = __reduce_min_sync(0xffffffffu, max(limit_row - it.kv_begin, 0) / kTile);
+        const int ragged_tile = ((it.kv_end - it.kv_begin) % kTile) ? n_tiles - 1 : -1;   // only a last tile can end early
+        // Everything that depends on the tile number is carried along instead of recomputed (the two warps of a
+        // sub-partition share its issue slots with each other and with a producer or MMA warp: instructions count).
+        int b = g_tile % kRing;                                   // S buffer of the tile
+        uint32_t b_phase = (g_tile / kRing) & 1;
+        uint32_t par = g_tile & 1;                                // mailbox slot of the tile's post
+        uint32_t tag = ((g_tile >> 1) & 1u) + 1u;                 // tag of the tile's post
+        uint32_t tag_prev = (((g_tile - 1) >> 1) & 1u) + 1u;      // tag of the previous tile's post (slot par ^ 1)
+        const uint32_t xm_own = smem_u32(&C.xmax[0][hf][row]), xm_oth = smem_u32(&C.xmax[0][hf ^ 1][row]);
         for (int j = 0; j < n_tiles; ++j) {
           const uint32_t gj = g_tile + j;
-          const int b = gj % kRing;
-          const uint32_t s_col = kColS + b * kTile;
-          // (no vote and no early exit here: after a wait has run out the CTA is aborting, the later waits fail fast
-          // and the thread runs the rest of the item on whatever it finds; `ok` keeps the result from being written)
-          if (!mbar_wait(&C.s_full[b], (gj / kRing) & 1, abort_flag)) ok = false;
+          const uint32_t s_col = kColS + b * kTile + hf * 64;     // this thread's 64 scores; its P goes over the first 32
+          if (!mbar_wait(&C.s_full[b], b_phase, abort_flag)) ok = false;
           tc_fence_after();
-          // the second half of the scores is fetched while the exponentials of the first half are computed
-          uint32_t sr[kTile];
+          uint32_t sr[64];
           tmem_ld32(tmem + lane_base + s_col, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
-          tmem_ld32(tmem + lane_base + s_col + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
           tmem_wait_ld();
-          tmem_ld32(tmem + lane_base + s_col + 64, *reinterpret_cast<uint32_t(*)[32]>(&sr[64]));
-          tmem_ld32(tmem + lane_base + s_col + 96, *reinterpret_cast<uint32_t(*)[32]>(&sr[96]));
+          tmem_ld32(tmem + lane_base + s_col + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
 
-          const int pos0 = it.kv_begin + j * kTile;
           const bool masked = j >= first_masked_tile;             // warp-uniform
-          if (masked) {                                           // causal tail or end of the source
+          bool second_in = false;
+          if (masked || j == 0) {
             tmem_wait_ld();
-            tmem_pin32(*reinterpret_cast<uint32_t(*)[32]>(&sr[64]));
-            tmem_pin32(*reinterpret_cast<uint32_t(*)[32]>(&sr[96]));
-            const int nvis = limit_row - pos0;                    // visible columns of this tile for this row
+            tmem_pin32(*reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
+            second_in = true;
+            if (masked) {
+              const int nvis = limit_row - (it.kv_begin + j * kTile + hf * 64);   // visible ones of this thread's columns
 #pragma unroll
-            for (int c = 0; c < kTile; ++c)
-              if (c >= nvis) sr[c] = 0xff800000u;                 // -inf
+              for (int c = 0; c < 64; ++c)
+                if (c >= nvis) sr[c] = 0xff800000u;               // -inf
+            }
           }
-          // Reference maximum, one tile behind: the exponentials of this tile are taken relative to the reference m
-          // that the previous tiles produced, so they do not have to wait for this tile's own maximum, which is
-          // computed alongside them (the SFU pipe bounds the loop; the FMNMX are free) and only decides the
-          // reference of the NEXT tile (when it exceeds m by more than 2^kLazyLog2, so O is rarely rescaled).
-          // out = O / l and lse = m*scale + ln l hold for any m; only the fp32 range limits how far a score may
-          // exceed the reference, hence the exact fallback below when a tile jumps by more than 2^kJumpLog2 (always
-          // the case for the first visible key, where m = -inf).
+          // ---- reference of this tile --------------------------------------------------------------------------------
           float alpha = 1.f;
-          if (m_next != m) {                                      // decided by the previous tile
-            alpha = ex2((m - m_next) * cl2);
-            m = m_next;
-            l *= alpha;
-          }
-          if (j == 0) {                                           // no reference yet: take this tile's exact maximum first
-            tmem_wait_ld();                                       // (instead of exponentials that the fallback would redo)
-            tmem_pin32(*reinterpret_cast<uint32_t(*)[32]>(&sr[64]));
-            tmem_pin32(*reinterpret_cast<uint32_t(*)[32]>(&sr[96]));
+          if (j == 0) {                                           // exact maximum of the first tile, both halves
             float e4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-            for (int c = 0; c < kTile; c += 2)
+            for (int c = 0; c < 64; c += 2)
               e4[(c >> 1) & 3] = max3(e4[(c >> 1) & 3], __uint_as_float(sr[c]), __uint_as_float(sr[c + 1]));
-            const float mxe = fmaxf(fmaxf(e4[0], e4[1]), fmaxf(e4[2], e4[3]));
-            if (mxe > -INFINITY) { m = mxe; m_next = mxe; }
+            const float mine = fmaxf(fmaxf(e4[0], e4[1]), fmaxf(e4[2], e4[3]));
+            uint32_t (*xch)[128] = C.xmax[par ^ 1];               // idle until the post of tile gj + 1
+            xch[hf][row] = __float_as_uint(mine);
+            pair_barrier();
+            const float mxe = fmaxf(mine, __uint_as_float(xch[hf ^ 1][row]));
+            m = mxe > -INFINITY ? mxe : 0.f;
+            pair_barrier();
+            xch[hf][row] = 0u;
+          } else {                                                // lagged: the sampled maxima of the previous tile
+            const uint32_t src = xm_oth + (par ^ 1u) * (2 * 128 * 4);
+            uint32_t other = ld_shared_volatile(src);
+            if ((other & 3u) != tag_prev) {                       // the other half is still inside the previous tile
+              const long long t0 = clock64();
+              while (((other = ld_shared_volatile(src)) & 3u) != tag_prev) {
+                if (*abort_flag || clock64() - t0 > kWaitCycles) { *abort_flag = 1; ok = false; break; }
+              }
+            }
+            const float mx_prev = fmaxf(__uint_as_float(own_post & ~3u), __uint_as_float(other & ~3u));
+            if (mx_prev > m + lazy_raw) {
+              alpha = ex2((m - mx_prev) * cl2);
+              m = mx_prev;
+              l *= alpha;
+            }
           }
-          float mc = m == -INFINITY ? 0.f : m * cl2;
-          // Every instruction of this loop costs an issue slot that the SFU does not hide (an ex2 holds the
-          // sub-partition for 8 clocks and the rest adds to it), so the scaling and the row sum work on fp32 pairs.
+          const float mc = m * cl2;
           const f32x2 cl2_2 = pack2(cl2, cl2);
-          f32x2 nmc2 = pack2(-mc, -mc);
+          const f32x2 nmc2 = pack2(-mc, -mc);
           f32x2 sum2[2] = {pack2(0.f, 0.f), pack2(0.f, 0.f)};
           float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-          uint32_t pr[kTile / 2];
+          uint32_t pr[32];
 #pragma unroll
-          for (int hf = 0; hf < 2; ++hf) {
-            if (hf == 1) {
-              tmem_wait_ld();                                     // (no-op when the mask path has waited already)
-              tmem_pin32(*reinterpret_cast<uint32_t(*)[32]>(&sr[64]));
-              tmem_pin32(*reinterpret_cast<uint32_t(*)[32]>(&sr[96]));
+          for (int part = 0; part < 2; ++part) {
+            if (part == 1 && !second_in) {
+              tmem_wait_ld();
+              tmem_pin32(*reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
             }
 #pragma unroll
-            for (int c = hf * 64; c < hf * 64 + 64; c += 2) {
+            for (int c = part * 32; c < part * 32 + 32; c += 2) {
               const float s0 = __uint_as_float(sr[c]), s1 = __uint_as_float(sr[c + 1]);
               float x0, x1;
               unpack2(fma2(pack2(s0, s1), cl2_2, nmc2), x0, x1);
@@ -324,78 +374,51 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
           float sum4[4];
           unpack2(sum2[0], sum4[0], sum4[1]);
           unpack2(sum2[1], sum4[2], sum4[3]);
-          // mx: maximum of a sample of the columns (enough to move the reference lazily).  A score far above the
-          // reference shows in the row sum of the tile instead, which costs nothing to test.
-          float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+          const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
           const float tile_sum = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
-          const bool jump = m == -INFINITY || !(tile_sum <= jump_sum);   // no reference yet, or beyond 2^kJumpLog2 / inf / NaN
-          const int n_keys = min(kTile, it.kv_end - pos0);
-          // one vote covers every rare path of a tile: exact fallback, O rescale, ragged end of the source
-          const bool rare = __any_sync(0xffffffffu, jump || (alpha != 1.f && j > 0)) || n_keys < kTile;
-          if (rare && __any_sync(0xffffffffu, jump)) {
-            if (jump) {                                           // exact path: this tile's own maximum is the reference
+          // post this tile's sampled maximum for the other half (finite or -inf; the tag marks the tile)
+          own_post = (__float_as_uint(mx) & ~3u) | tag;
+          st_shared(xm_own + par * (2 * 128 * 4), own_post);
+          if (!(tile_sum <= jump_sum)) C.overflow[slot] = 1;     // beyond the lagged reference's range: exact pass needed
+          l += tile_sum;
+          const bool ragged = j == ragged_tile;
+          const bool rare = __any_sync(0xffffffffu, alpha != 1.f && j > 0) || ragged;
+          if (rare && hf == 0) {                                  // the first half's warps own O and the V tail
+            if (__any_sync(0xffffffffu, alpha != 1.f && j > 0)) { // rescale O (warp-collective TMEM access)
+              ok = mbar_wait(&C.pv_done[(gj - 1) % kRing], ((gj - 1) / kRing) & 1, abort_flag) && ok;
+              tc_fence_after();
+#pragma unroll 1
+              for (int c0 = 0; c0 < kHeadDim; c0 += 32) {
+                uint32_t o0[32];
+                tmem_ld32(tmem + lane_base + kColO + c0, o0);
+                tmem_wait_ld();
 #pragma unroll
-              for (int c = 0; c < kTile; c += 2)
-                mx4[(c >> 1) & 3] = max3(mx4[(c >> 1) & 3], __uint_as_float(sr[c]), __uint_as_float(sr[c + 1]));
-              mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-            }
-            if (jump && mx > -INFINITY) {
-              const float a2 = ex2((m - mx) * cl2);               // 0 when the row had no visible key so far
-              alpha *= a2;
-              l *= a2;
-              m = mx;
-              mc = m * cl2;
-              sum4[0] = sum4[1] = sum4[2] = sum4[3] = 0.f;
-#pragma unroll
-              for (int c = 0; c < kTile; c += 2) {
-                const float p0 = ex2(__uint_as_float(sr[c]) * cl2 - mc);
-                const float p1 = ex2(__uint_as_float(sr[c + 1]) * cl2 - mc);
-                sum4[(c >> 1) & 3] += p0 + p1;
-                pr[c >> 1] = pack_bf16_rn(p0, p1);
+                for (int x = 0; x < 32; ++x) o0[x] = __float_as_uint(__uint_as_float(o0[x]) * alpha);
+                tmem_st32(tmem + lane_base + kColO + c0, o0);
               }
             }
-          }
-          l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
-          m_next = mx > m + lazy_raw ? mx : m;
-          const bool move = alpha != 1.f;
-
-          if (rare && __any_sync(0xffffffffu, move && j > 0)) {   // rescale O (warp-collective TMEM access)
-            ok = mbar_wait(&C.pv_done[(gj - 1) % kRing], ((gj - 1) / kRing) & 1, abort_flag);   // PV(j-1) has landed in O
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            tc_fence_after();
-#pragma unroll
-            for (int c0 = 0; c0 < kHeadDim; c0 += 32) {
-              uint32_t o0[32];
-              tmem_ld32(tmem + lane_base + kColO + c0, o0);
-              tmem_wait_ld();
-#pragma unroll
-              for (int x = 0; x < 32; ++x) o0[x] = __float_as_uint(__uint_as_float(o0[x]) * alpha);
-              tmem_st32(tmem + lane_base + kColO + c0, o0);
-            }
-            tmem_wait_st();
-          }
-          // ---- last tile of a source that ends inside a page / inside the tile: zero the V rows past the end ---
-          if (n_keys < kTile) {
-            const int s = gj % kStagesV;
-            ok = mbar_wait(&C.v_full[s], (gj / kStagesV) & 1, abort_flag);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            uint8_t* vs = smem + kOffV + s * kStageBytes;
-            const int n_chunks = (kTile - n_keys) * 16;           // 16-byte chunks to clear (both halves)
-            for (int x = tid; x < n_chunks; x += kSoftmaxWarps * 32) {
-              const int r = n_keys + (x >> 4), cc = x & 15;
-              *reinterpret_cast<uint4*>(vs + (cc >> 3) * (kStageBytes / 2) + r * 128 + (cc & 7) * 16) = make_uint4(0, 0, 0, 0);
+            if (ragged) {                                         // zero the V rows past the end of the source
+              const int n_keys = it.kv_end - (it.kv_begin + j * kTile);
+              const int s = gj % kStagesV;
+              ok = mbar_wait(&C.v_full[s], (gj / kStagesV) & 1, abort_flag) && ok;
+              uint8_t* vs = smem + kOffV + s * kStageBytes;
+              const int n_chunks = (kTile - n_keys) * 16;         // 16-byte chunks to clear (both halves)
+              for (int x = row; x < n_chunks; x += 128) {
+                const int r = n_keys + (x >> 4), cc = x & 15;
+                *reinterpret_cast<uint4*>(vs + (cc >> 3) * (kStageBytes / 2) + r * 128 + (cc & 7) * 16) = make_uint4(0, 0, 0, 0);
+              }
+              fence_proxy_async_smem();
             }
           }
-          // ---- P (bf16 pairs) over the first 64 columns of its own S buffer: the A operand of PV, read from TMEM ------
-#pragma unroll
-          for (int c0 = 0; c0 < kTile / 2; c0 += 32)
-            tmem_st32(tmem + lane_base + s_col + c0, *reinterpret_cast<uint32_t(*)[32]>(&pr[c0]));
+          // ---- P (bf16 pairs) over the first 32 of this thread's own 64 score columns -------------------------------
+          tmem_st32(tmem + lane_base + s_col, pr);
           tmem_wait_st();
-          if (n_keys < kTile) fence_proxy_async_smem();           // the V rows cleared above
           tc_fence_before();
           mbar_arrive(&C.p_full[b]);
+          if (++b == kRing) { b = 0; b_phase ^= 1u; }
+          tag_prev = tag;
+          if (par) tag ^= 3u;                                     // (the tag changes with every second tile: 1 <-> 2)
+          par ^= 1u;
         }
         ok = __all_sync(0xffffffffu, ok);
         if (ok) {
@@ -404,14 +427,19 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
           tc_fence_after();
         }
       }
-      // ---- epilogue --------------------------------------------------------------------------------------------------
+      // ---- epilogue: the two halves add their row sums; each writes 64 output columns ---------------------------------
+      C.xmax[0][hf][row] = __float_as_uint(l);                  // (every tile of the item is behind both halves here)
+      pair_barrier();
+      const float l_all = l + __uint_as_float(C.xmax[0][hf ^ 1][row]);
+      pair_barrier();
+      C.xmax[0][hf][row] = 0u;
       if (ok) {
-        const float inv = l > 0.f ? 1.f / l : 0.f;
-        const float lse = l > 0.f ? m * P.scale + __logf(l) : -INFINITY;
+        const float inv = l_all > 0.f ? 1.f / l_all : 0.f;
+        const float lse = l_all > 0.f ? m * P.scale + __logf(l_all) : -INFINITY;
         const bool final_out = it.slot_off < 0;
-        const int64_t slot = final_out ? 0 : static_cast<int64_t>(row_valid ? P.dec_slot_base[dec] : 0) + it.slot_off;
+        const int64_t slot_row = final_out ? 0 : static_cast<int64_t>(row_valid ? P.dec_slot_base[dec] : 0) + it.slot_off;
 #pragma unroll
-        for (int c0 = 0; c0 < kHeadDim; c0 += 32) {
+        for (int c0 = hf * 64; c0 < hf * 64 + 64; c0 += 32) {
           uint32_t orow[32];
           __syncwarp();                                         // the TMEM load below is warp-collective
           if (n_tiles > 0) {
@@ -433,7 +461,7 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
               st_global_32B(dst + 16 * x, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]);
             }
           } else {
-            float* dst = P.part_o + (slot * P.Hq + h) * kHeadDim + c0;
+            float* dst = P.part_o + (slot_row * P.Hq + h) * kHeadDim + c0;
 #pragma unroll
             for (int x = 0; x < 4; ++x) {
               uint32_t w[8];
@@ -443,9 +471,9 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
             }
           }
         }
-        if (row_valid) {
+        if (row_valid && hf == 0) {
           if (final_out) { if (P.lse) P.lse[q_row * P.Hq + h] = lse; }
-          else P.part_lse[slot * P.Hq + h] = lse;
+          else P.part_lse[slot_row * P.Hq + h] = lse;
         }
       }
     } else if (warp < kSoftmaxWarps + 2) {
@@ -616,8 +644,8 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
           const uint64_t v_desc = smem_desc_advance(v_desc0, static_cast<uint32_t>(s) * kStageBytes);
           const uint32_t o_tmem = tmem + kColO, p_tmem = tmem + kColS + b * kTile;
 #pragma unroll
-          for (int kk = 0; kk < kTile / 16; ++kk)
-            mma_bf16_ts(o_tmem, p_tmem + kk * 8, smem_desc_advance(v_desc, kk * 2048), idesc_pv,
+          for (int kk = 0; kk < kTile / 16; ++kk)       // P of keys 0..63 at columns 0..31, of keys 64..127 at 64..95
+            mma_bf16_ts(o_tmem, p_tmem + (kk >> 2) * 64 + (kk & 3) * 8, smem_desc_advance(v_desc, kk * 2048), idesc_pv,
                         (j > 0 || kk > 0) ? 1u : 0u);
           mma_commit(&C.v_empty[s]);
           mma_commit(&C.pv_done[b]);
@@ -629,6 +657,14 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    // Exact second pass: the exponentials of some half-row overflowed the range of the lagged reference (scores that
+    // rise by more than 2^40 from one tile to the next; the tensor-core pass has then written garbage for the
+    // item).  All twelve warps recompute the item's rows on the CUDA cores, one row per warp and key by key.
+    if (C.overflow[slot]) {
+      exact_second_pass(P, &C.item[slot], warp, lane);
+      __syncthreads();
+      if (tid == 0) C.overflow[slot] = 0;
+    }
     g_tile += n_tiles;
     if (n_tiles > 0) {
       ++q_uses;
@@ -648,13 +684,13 @@ tile_items_umma_deep_kernel(const __grid_constant__ CUtensorMap tmap_k, const __
   if (warp == kSoftmaxWarps) tmem_dealloc(tmem, kTmemCols);
 }
 
-}  // namespace deep
+}  // namespace split
 
-int32_t launch_tile_items_umma_deep(const Params& P, cudaStream_t st, int sm_count) {
-  using namespace deep;
+int32_t launch_tile_items_umma_split(const Params& P, cudaStream_t st, int sm_count) {
+  using namespace split;
   static bool configured = false;
   if (!configured) {
-    if (cudaFuncSetAttribute(tile_items_umma_deep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kUmmaSmem) !=
+    if (cudaFuncSetAttribute(tile_items_umma_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kUmmaSmem) !=
         cudaSuccess) {
       (void)cudaGetLastError();
       return SS_ERR_CUDA;
@@ -673,7 +709,7 @@ int32_t launch_tile_items_umma_deep(const Params& P, cudaStream_t st, int sm_cou
   if (!tmap::encode_q_bf16(&tq, P.q, static_cast<uint64_t>(P.Hq), static_cast<uint64_t>(q_rows > 0 ? q_rows : 1),
                            static_cast<uint32_t>(P.G), static_cast<uint32_t>(P.tok_per_tile)))
     return SS_ERR_CUDA;
-  SS_LAUNCH(tile_items_umma_deep_kernel, sm_count, kUmmaThreads, kUmmaSmem, st, tk, tv, tq, P);
+  SS_LAUNCH(tile_items_umma_split_kernel, sm_count, kUmmaThreads, kUmmaSmem, st, tk, tv, tq, P);
   return SS_OK;
 }
 
