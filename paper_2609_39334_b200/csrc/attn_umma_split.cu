@@ -44,7 +44,7 @@ namespace split {
 constexpr int kSoftmaxWarps = 8;               // two warps per TMEM lane quarter: each takes 64 of a row's 128 scores
 constexpr int kUmmaThreads = (kSoftmaxWarps + 4) * 32;
 constexpr int kTile = 128;                     // keys per tile (two of the planner's 64-key tiles)
-constexpr int kStageBytes = kTile * 256;       // one K or V tile: [2 halves of 64 dims][kTile rows][128 B]
+constexpr int kStageBytes = kTile * 256;       // one K or V tile: [16 groups of 8 keys][2 halves of 64 dims][8 rows][128 B]
 constexpr int kStagesK = 3;
 constexpr int kStagesV = 2;                    // V is consumed a softmax later than K: two stages are enough
 constexpr int kRing = 3;                       // S/P buffers
@@ -405,7 +405,7 @@ tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const _
               const int n_chunks = (kTile - n_keys) * 16;         // 16-byte chunks to clear (both halves)
               for (int x = row; x < n_chunks; x += 128) {
                 const int r = n_keys + (x >> 4), cc = x & 15;
-                *reinterpret_cast<uint4*>(vs + (cc >> 3) * (kStageBytes / 2) + r * 128 + (cc & 7) * 16) = make_uint4(0, 0, 0, 0);
+                *reinterpret_cast<uint4*>(vs + (r >> 3) * 2048 + (cc >> 3) * 1024 + (r & 7) * 128 + (cc & 7) * 16) = make_uint4(0, 0, 0, 0);
               }
               fence_proxy_async_smem();
             }
@@ -561,8 +561,7 @@ tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const _
 #pragma unroll
               for (int pg = 0; pg < kTile / kPage; ++pg) {
                 if (pg < n_pages) {
-                  tma_load_2d(dst + pg * 2048, tm, 0, y[pg], &full[s]);
-                  tma_load_2d(dst + kStageBytes / 2 + pg * 2048, tm, 64, y[pg], &full[s]);
+                  tma_load_4d(dst + pg * 4096, tm, 0, 0, 0, y[pg] >> 3, &full[s]);   // the whole (page, head) block
                 }
               }
               if (++s == n_stages) { s = 0; ++u; }
@@ -606,7 +605,7 @@ tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const _
       if (n_tiles > 0 && elect_one()) {                          // (elected, not `lane == 0`: see the producers)
         constexpr uint32_t idesc_qk = instr_desc_bf16(128, kTile, false);
         const uint64_t q_desc0 = smem_desc_sw128(smem_u32(smem + kOffQ + slot * 32768), 0, 1024);
-        const uint64_t k_desc0 = smem_desc_sw128(smem_u32(smem + kOffK), 0, 1024);
+        const uint64_t k_desc0 = smem_desc_sw128(smem_u32(smem + kOffK), 0, 2048);   // 8-key groups 2048 B apart
         bool ok = it.kind == kItemChain ? mbar_wait(&C.q_full_tma, q_uses_tma & 1, abort_flag)
                                         : mbar_wait(&C.q_full, (q_uses - q_uses_tma) & 1, abort_flag);
         for (int j = 0; j < n_tiles && ok; ++j) {
@@ -622,7 +621,7 @@ tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const _
 #pragma unroll
           for (int kk = 0; kk < 8; ++kk)
             mma_bf16_ss(d_tmem, smem_desc_advance(q_desc0, (kk >> 2) * 16384 + (kk & 3) * 32),
-                        smem_desc_advance(k_desc, (kk >> 2) * (kStageBytes / 2) + (kk & 3) * 32), idesc_qk,
+                        smem_desc_advance(k_desc, (kk >> 2) * 1024 + (kk & 3) * 32), idesc_qk,
                         kk > 0 ? 1u : 0u);
           mma_commit(&C.k_empty[s]);
           mma_commit(&C.s_full[b]);
@@ -632,7 +631,7 @@ tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const _
       // =================================================== O += P V issuer =====================================
       if (n_tiles > 0 && elect_one()) {
         constexpr uint32_t idesc_pv = instr_desc_bf16(128, kHeadDim, true);
-        const uint64_t v_desc0 = smem_desc_sw128(smem_u32(smem + kOffV), kStageBytes / 2, 1024);
+        const uint64_t v_desc0 = smem_desc_sw128(smem_u32(smem + kOffV), 1024, 2048);   // dims 64..127 1024 B on, 8-key groups 2048 B apart
         bool ok = true;
         for (int j = 0; j < n_tiles && ok; ++j) {
           const uint32_t gj = g_tile + j;
@@ -645,7 +644,7 @@ tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const _
           const uint32_t o_tmem = tmem + kColO, p_tmem = tmem + kColS + b * kTile;
 #pragma unroll
           for (int kk = 0; kk < kTile / 16; ++kk)       // P of keys 0..63 at columns 0..31, of keys 64..127 at 64..95
-            mma_bf16_ts(o_tmem, p_tmem + (kk >> 2) * 64 + (kk & 3) * 8, smem_desc_advance(v_desc, kk * 2048), idesc_pv,
+            mma_bf16_ts(o_tmem, p_tmem + (kk >> 2) * 64 + (kk & 3) * 8, smem_desc_advance(v_desc, kk * 4096), idesc_pv,
                         (j > 0 || kk > 0) ? 1u : 0u);
           mma_commit(&C.v_empty[s]);
           mma_commit(&C.pv_done[b]);
@@ -686,8 +685,13 @@ tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const _
 
 }  // namespace split
 
+int32_t launch_tile_items_umma(const Params& P, cudaStream_t st, int sm_count);   // the 64-key kernel (attn_umma.cu)
+
 int32_t launch_tile_items_umma_split(const Params& P, cudaStream_t st, int sm_count) {
   using namespace split;
+  // One bulk-tensor copy per (page, kv head) block needs the blocks to start on 8-row boundaries of the pool (rows of
+  // 256 bytes); any other pool layout goes to the kernel that copies the two 64-dim halves of a block separately.
+  if (P.page_stride % 1024 || P.head_stride % 1024) return launch_tile_items_umma(P, st, sm_count);
   static bool configured = false;
   if (!configured) {
     if (cudaFuncSetAttribute(tile_items_umma_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kUmmaSmem) !=
@@ -700,8 +704,8 @@ int32_t launch_tile_items_umma_split(const Params& P, cudaStream_t st, int sm_co
   const int64_t rows = ((P.num_pages > 0 ? P.num_pages - 1 : 0) * P.page_stride + (P.Hkv - 1) * P.head_stride) / 128 + kPage;
   if (rows >= 0x7fffffffLL) return SS_ERR_UNSUPPORTED;
   CUtensorMap tk, tv;
-  if (!tmap::encode_2d_bf16(&tk, P.k_pool, kHeadDim, static_cast<uint64_t>(rows), kHeadDim * 2, kPage) ||
-      !tmap::encode_2d_bf16(&tv, P.v_pool, kHeadDim, static_cast<uint64_t>(rows), kHeadDim * 2, kPage))
+  if (!tmap::encode_kv_block_bf16(&tk, P.k_pool, static_cast<uint64_t>(rows)) ||
+      !tmap::encode_kv_block_bf16(&tv, P.v_pool, static_cast<uint64_t>(rows)))
     return SS_ERR_CUDA;
   // one CTA per SM: the kernel takes all 512 TMEM columns and most of the shared memory
   CUtensorMap tq;

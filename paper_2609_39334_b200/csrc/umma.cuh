@@ -88,6 +88,12 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* t
       ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(smem_u32(bar))
       : "memory");
 }
+__device__ __forceinline__ void tma_load_4d(void* smem_dst, const CUtensorMap* tmap, int x, int y, int z, int w, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+      ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(z), "r"(w), "r"(smem_u32(bar))
+      : "memory");
+}
 __device__ __forceinline__ void tma_load_3d(void* smem_dst, const CUtensorMap* tmap, int x, int y, int z, uint64_t* bar) {
   asm volatile(
       "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
@@ -217,6 +223,7 @@ namespace tmap {
 bool encode_2d_bf16(CUtensorMap* out, const void* base, uint64_t row_elems, uint64_t rows, uint64_t pitch_bytes,
                     uint32_t box_rows);
 // 3-D bf16 tensor [tokens_total][q_heads][128], loaded in boxes of 64 dims x `heads` x `tokens` with the 128-byte swizzle.
+bool encode_kv_block_bf16(CUtensorMap* out, const void* base, uint64_t rows);
 bool encode_q_bf16(CUtensorMap* out, const void* base, uint64_t q_heads, uint64_t tokens_total, uint32_t heads,
                    uint32_t tokens);
 }  // namespace tmap

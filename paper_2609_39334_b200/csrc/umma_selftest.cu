@@ -39,6 +39,24 @@ bool encode_2d_bf16(CUtensorMap* out, const void* base, uint64_t row_elems, uint
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// K / V pool viewed as rows of 128 bf16 (256 bytes).  One box = 16 consecutive rows (one page of one kv head) x all
+// 128 dims, delivered as the tensor-core operand layout wants it: for each group of 8 rows, first the 8 x 128-byte
+// rows of dims 0..63 (one 1024-byte swizzle atom), then those of dims 64..127.  Dimensions, innermost first:
+// 64 dims (2 B apart), 8 rows (256 B), 2 halves of the row (128 B), groups of 8 rows (2048 B); the coordinate of a box
+// is (0, 0, 0, first row / 8).  The strides are not monotonic (the third is smaller than the second): the rows of a
+// half are gathered before the halves are.
+bool encode_kv_block_bf16(CUtensorMap* out, const void* base, uint64_t rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[4] = {64, 8, 2, rows / 8};
+  const cuuint64_t strides[3] = {256, 128, 2048};
+  const cuuint32_t box[4] = {64, 8, 2, 2};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // Query rows: q viewed as [token][q head][128] bf16; boxes of 64 dims x `heads` heads x `tokens` tokens land in shared
 // memory as consecutive 128-byte rows (token-major, then head) with the 128-byte swizzle.
 bool encode_q_bf16(CUtensorMap* out, const void* base, uint64_t q_heads, uint64_t tokens_total, uint32_t heads,
