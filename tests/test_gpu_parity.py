@@ -586,3 +586,28 @@ def test_attention_score_jumps_between_tiles(mode, flags):
     fin = np.isfinite(l_ref)
     # lse is a raw score here (hundreds): compare relative to its size
     assert np.abs(r["lse"][fin] - l_ref[fin]).max() <= 2e-3 * max(1.0, np.abs(l_ref[fin]).max())
+
+
+def test_attention_pool_blocks_off_the_8_row_grid():
+    """A K / V pool whose (page, head) blocks are 17 rows apart (strides that are multiples of 128 elements, as the
+    interface asks, but not of 8 rows): the default tile kernel's one-copy-per-block path cannot address it and the
+    call must take the other tensor-core kernel, with the same results."""
+    name, Hq, Hkv, levels, fanout, problems, leaf, qfn, dup = SHAPES[1]
+    w = synth.build_tree_workload(name, 4321, Hq, Hkv, levels, fanout, problems, leaf, qfn, dup_frac=dup)
+    pipe = DevicePipeline(w, DEV, attn_flags=B.SS_FLAG_VALIDATE)
+    pool = pipe.kv_pool                                         # [page][2][Hkv][16][128]
+    padded = torch.zeros((pool.shape[0], 2, Hkv, 17, 128), dtype=torch.bfloat16, device=pool.device)
+    padded[:, :, :, :16] = pool
+    padded[:, :, :, 16] = float("nan")                          # the padding row must never be read
+    d = pipe.desc
+    blk = Hkv * 17 * 128
+    d.k_pool = padded.data_ptr()
+    d.v_pool = padded.data_ptr() + blk * 2
+    d.kv_page_stride, d.kv_head_stride, d.kv_token_stride = 2 * blk, 17 * 128, 128
+    pipe.attn_ws = B.alloc_workspace(B.ss_tree_attention_workspace_bytes(d), pool.device)
+    pipe.dedup()
+    pipe.compact_unique()
+    pipe.attention()
+    r = pipe.results()
+    ref = oracle.dedup(w.tok_ids, w.tok_offsets, w.ctx_key, w.slot_in)
+    check_attention(r, w, ref, max_paths=64)
