@@ -368,7 +368,7 @@ tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const _
               const float p0 = ex2(x0), p1 = ex2(x1);
               sum2[(c >> 1) & 1] = add2(sum2[(c >> 1) & 1], pack2(p0, p1));
               pr[c >> 1] = pack_bf16_rn(p0, p1);
-              if ((c & 6) == 0) mx4[(c >> 3) & 3] = max3(mx4[(c >> 3) & 3], s0, s1);   // every fourth pair
+              if ((c & 14) == 0) mx4[(c >> 4) & 3] = max3(mx4[(c >> 4) & 3], s0, s1);   // every eighth pair
             }
           }
           float sum4[4];
