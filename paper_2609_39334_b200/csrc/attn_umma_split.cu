@@ -341,7 +341,8 @@ tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const _
                 if (*abort_flag || clock64() - t0 > kWaitCycles) { *abort_flag = 1; ok = false; break; }
               }
             }
-            const float mx_prev = fmaxf(__uint_as_float(own_post & ~3u), __uint_as_float(other & ~3u));
+            // (the tag bits stay in: both threads of the row compare the same two words)
+            const float mx_prev = fmaxf(__uint_as_float(own_post), __uint_as_float(other));
             if (mx_prev > m + lazy_raw) {
               alpha = ex2((m - mx_prev) * cl2);
               m = mx_prev;
