@@ -383,8 +383,9 @@ tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const _
           if (!(tile_sum <= jump_sum)) C.overflow[slot] = 1;     // beyond the lagged reference's range: exact pass needed
           l += tile_sum;
           const bool ragged = j == ragged_tile;
-          const bool rare = __any_sync(0xffffffffu, alpha != 1.f && j > 0) || ragged;
-          if (rare && hf == 0) {                                  // the first half's warps own O and the V tail
+          // (only the first half's warps vote: they own O and the V tail, and a vote per tile in every warp costs 3 %)
+          const bool rare = hf == 0 && (__any_sync(0xffffffffu, alpha != 1.f && j > 0) || ragged);
+          if (rare) {
             if (__any_sync(0xffffffffu, alpha != 1.f && j > 0)) { // rescale O (warp-collective TMEM access)
               ok = mbar_wait(&C.pv_done[(gj - 1) % kRing], ((gj - 1) / kRing) & 1, abort_flag) && ok;
               tc_fence_after();
