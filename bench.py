@@ -453,7 +453,7 @@ def main():
         host.synchronize()
         host.results(0)                                   # raises on a device-side error
         sync_all()
-        n_e2e = max(args.steps, 2 * args.e2e_depth)
+        n_e2e = max(2 * args.steps, 2 * args.e2e_depth)   # (twice K: the first and the last step copy one way only)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         cur = torch.cuda.current_stream(dev)
         e0.record(cur)
