@@ -30,6 +30,7 @@ UNIT = "tokens/s"
 WORKLOADS = {"c2": 2, "c3": 3, "c4": 4, "c5": 5}
 LV_SWEEP_TOKENS = [256, 512, 1024, 2048, 4096, 8192, 16384]
 L2_BYTES = 126 * 1024 * 1024
+MIN_ORACLE_SAMPLE = 128             # unique paths in the oracle's bounded sample
 NOMINAL_HBM_GBS = 8000.0            # vendor figures, reported beside the measured peaks for context only
 NOMINAL_BF16_TFLOPS = 2250.0
 
@@ -149,14 +150,15 @@ def oracle_sample(w, seed=0):
     budget_pairs = 12.0 * cores * 0.7e9 / (2.0 * w.head_dim * w.num_q_heads)
     chosen, pairs = [], 0.0
     pools = [list(rng.permutation(ver)), list(rng.permutation(dec))]
-    while (pools[0] or pools[1]) and pairs < budget_pairs:
-        for pool in pools:
-            if pool:
-                p = int(pool.pop())
-                L = w.path_kv_len(p)
-                Tp = int(w.path_q_len[p])
-                pairs += Tp * L
-                chosen.append(p)
+    turn = 0
+    # one verification path, then three decode paths (a decode path costs 1/T of a verification path), until the
+    # budget is spent AND at least MIN_ORACLE_SAMPLE unique paths are in
+    while (pools[0] or pools[1]) and (pairs < budget_pairs or len(chosen) < MIN_ORACLE_SAMPLE):
+        pool = pools[0] if (turn % 4 == 0 and pools[0]) or not pools[1] else pools[1]
+        turn += 1
+        p = int(pool.pop())
+        pairs += int(w.path_q_len[p]) * w.path_kv_len(p)
+        chosen.append(p)
     return np.asarray(sorted(chosen), np.int64)
 
 

@@ -67,7 +67,7 @@ int32_t ss_last_device_status(const void* workspace, void* stream, int32_t* out_
 /* =========================================================================================================
  * ss_dedup_paths - computation deduplication.
  *
- * Paper: Section "Computation Deduplication" - candidates "with identical input sequences" share one
+ * Paper: Section "Computation Deduplication" - candidates whose input sequences are identical share one
  * forward pass; the number of logical candidates a sequence stands for is its "potential" size, and
  * sampled continuations are grouped by equality with one child per group whose potential is the group's
  * cardinality (worked example: three equal samples and one different -> potentials 3 and 1).
@@ -152,7 +152,7 @@ int32_t ss_dedup_paths_static(const int32_t* tok_ids, const int64_t* tok_offsets
  *
  * Paper: the serving substrate of Section "Experimental Setup" (paged attention, prefix KV caching and
  * sharing, fused attention kernels), used for the decode phase of expansion (Section "LLM Inference and
- * Serving") and for verification, which "is a prefill-only workload" over short steps (Section "Lazy
+ * Serving") and for verification, which only prefills short steps (no decoding) (Section "Lazy
  * Verification").  The paper prints no formula; the operation is standard softmax attention:
  *
  *   for path p with KV sequence = concatenation of its nodes root -> leaf (length L), step length T:
@@ -179,7 +179,8 @@ int32_t ss_dedup_paths_static(const int32_t* tok_ids, const int64_t* tok_offsets
  *
  * q   bf16 [total_q][Hq][128], rows of path p are q_offsets[p] .. q_offsets[p+1]-1 (or start at q_src_offsets[p] in
  *     a larger array, see the descriptor), 16-byte aligned
- * out bf16 [total_q][Hq][128]   (fp32 accumulation, rounded to nearest even), 16-byte aligned
+ * out bf16 [total_q][Hq][128]   (fp32 accumulation, rounded to nearest even), 32-byte aligned (the tile kernel
+ *                               writes whole 32-byte sectors; any other alignment => SS_ERR_UNSUPPORTED)
  * lse fp32 [total_q][Hq]        or NULL
  *
  * Accuracy contract (inputs ~N(0,1) in bf16): |out - exact| <= 2e-2 max, 2e-3 mean; |lse - exact| <= 1e-3.
@@ -287,7 +288,7 @@ int32_t ss_early_prune(const float* scores, const uint8_t* verified, const int32
  * ss_branch_sample - the draws of on-demand branching.
  *
  * Paper: Section "Computation Deduplication" - a sequence with potential size n runs one forward pass and then
- * samples n next tokens "as independent trials from the same distribution"; equal samples are grouped and every
+ * draws n next tokens independently from that one distribution; equal samples are grouped and every
  * group becomes one child sequence whose potential size is the group's cardinality.  This call does the sampling;
  * the grouping is ss_dedup_paths on the (sequence, token) pairs it returns (tok_ids = tokens_out with one token per
  * path, ctx_key = seq_out): multiplicity_out are then the children's potential sizes.  (The paper batches the

@@ -5,7 +5,7 @@
 // called from it; only the test-suite, the smoke check and the benchmark's cpu_baseline / reference arm may
 // load it.  Everything is host memory; floating point is fp64.
 //
-//   ss_oracle_dedup           Computation deduplication: candidates "with identical input sequences" form one
+//   ss_oracle_dedup           Computation deduplication: candidates whose input sequences are identical form one
 //                             group that is computed once; the group's size is the sequence's "potential"
 //                             (paper, Section "Computation Deduplication").  Plain definition with std::map.
 //   ss_oracle_tree_attention  Softmax attention of every candidate path over its own root-to-leaf KV

@@ -85,7 +85,7 @@ static Layout carve(const ss_attn_desc_t* d, char* base, Params* P) {
   const int max_depth = d->max_depth > 0 ? d->max_depth : SS_MAX_DEPTH;
   const int64_t cap_dec = d->max_decode_paths > 0 ? (d->max_decode_paths < d->num_paths ? d->max_decode_paths : d->num_paths)
                                                   : d->num_paths;
-  const int target = 2 * 148;
+  const int target = 2 * sm_count_of_current_device();   // (the size query and the call must see the same device)
   Caps caps;
   caps.dec = static_cast<int32_t>(cap_dec);
   const int64_t stacked = static_cast<int64_t>(Hkv) * (cap_dec * max_depth / tpt + d->num_nodes) + target + Hkv * kMaxRootSplits;
@@ -156,7 +156,7 @@ extern "C" int32_t ss_tree_attention(const ss_attn_desc_t* d, void* workspace, s
     return SS_ERR_INVALID_ARG;
   if (d->total_q > 0 && (!d->q || !d->out)) return SS_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(d->k_pool) % 256 || reinterpret_cast<uintptr_t>(d->v_pool) % 256 ||
-      reinterpret_cast<uintptr_t>(d->q) % 16 || reinterpret_cast<uintptr_t>(d->out) % 16)
+      reinterpret_cast<uintptr_t>(d->q) % 16 || reinterpret_cast<uintptr_t>(d->out) % 32)
     return SS_ERR_UNSUPPORTED;
   if (d->total_q > 0x7fffffffLL / d->num_q_heads) return SS_ERR_UNSUPPORTED;   // row indices are int32
   if (d->q_src_offsets && (d->q_src_rows < 0 || d->q_src_rows > 0x7fffffffLL / d->num_q_heads)) return SS_ERR_INVALID_ARG;

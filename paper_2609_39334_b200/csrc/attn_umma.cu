@@ -436,9 +436,10 @@ tile_items_umma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_
 int g_tile_kernel_occupancy = 0;   // CTAs per SM reported by the occupancy query (diagnostics)
 
 int32_t launch_tile_items_umma(const Params& P, cudaStream_t st, int sm_count) {
-  static bool configured = false;
-  static int ctas_per_sm = 1;
-  if (!configured) {
+  static bool configured[kDeviceSlots] = {false};     // the attributes belong to the (function, device) pair
+  constexpr int ctas_per_sm = 2;                      // TMEM: 2 x 256 columns per SM; extra CTAs simply queue
+  const int dev_slot = current_device_slot();
+  if (dev_slot < 0 || !configured[dev_slot]) {
     if (cudaFuncSetAttribute(tile_items_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kUmmaSmem) !=
         cudaSuccess) {
       (void)cudaGetLastError();
@@ -455,8 +456,7 @@ int32_t launch_tile_items_umma(const Params& P, cudaStream_t st, int sm_count) {
       occ = 1;
     }
     g_tile_kernel_occupancy = occ;
-    ctas_per_sm = 2;                             // TMEM: 2 x 256 columns per SM; extra CTAs simply queue
-    configured = true;
+    if (dev_slot >= 0) configured[dev_slot] = true;
   }
   const int64_t rows = ((P.num_pages > 0 ? P.num_pages - 1 : 0) * P.page_stride + (P.Hkv - 1) * P.head_stride) / 128 + kPage;
   if (rows >= 0x7fffffffLL) return SS_ERR_UNSUPPORTED;

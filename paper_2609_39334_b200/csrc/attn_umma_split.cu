@@ -694,14 +694,15 @@ int32_t launch_tile_items_umma_split(const Params& P, cudaStream_t st, int sm_co
   // One bulk-tensor copy per (page, kv head) block needs the blocks to start on 8-row boundaries of the pool (rows of
   // 256 bytes); any other pool layout goes to the kernel that copies the two 64-dim halves of a block separately.
   if (P.page_stride % 1024 || P.head_stride % 1024) return launch_tile_items_umma(P, st, sm_count);
-  static bool configured = false;
-  if (!configured) {
+  static bool configured[kDeviceSlots] = {false};     // the attribute belongs to the (function, device) pair
+  const int dev_slot = current_device_slot();
+  if (dev_slot < 0 || !configured[dev_slot]) {
     if (cudaFuncSetAttribute(tile_items_umma_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kUmmaSmem) !=
         cudaSuccess) {
       (void)cudaGetLastError();
       return SS_ERR_CUDA;
     }
-    configured = true;
+    if (dev_slot >= 0) configured[dev_slot] = true;
   }
   const int64_t rows = ((P.num_pages > 0 ? P.num_pages - 1 : 0) * P.page_stride + (P.Hkv - 1) * P.head_stride) / 128 + kPage;
   if (rows >= 0x7fffffffLL) return SS_ERR_UNSUPPORTED;

@@ -43,6 +43,17 @@ bool pdl_enabled();
     }                                                                             \
   } while (0)
 
+// Function attributes and device properties are per device, so "done once" caches are arrays indexed by the current
+// device.  Returns the device's index, or -1 when it cannot be used as an index (the caller then skips its cache).
+// The host-side caches of the library (these, the launch counter, the event profiler) are not guarded by locks:
+// calls that share a device must come from one thread at a time.
+constexpr int kDeviceSlots = 64;
+inline int current_device_slot() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); return -1; }
+  return (dev >= 0 && dev < kDeviceSlots) ? dev : -1;
+}
+
 constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
 

@@ -77,6 +77,18 @@ def test_attention_descriptor_validation_on_host(lib):
     assert lib.ss_tree_attention(ctypes.byref(_desc()), None, ctypes.c_size_t(0), None) == B.SS_ERR_INVALID_ARG
 
 
+def test_attention_rejects_an_output_that_is_not_32_byte_aligned(lib):
+    """The tile kernel writes whole 32-byte sectors of `out`; a pointer that is only 16-byte aligned is refused on the
+    host, before anything is launched (the pointers below are never dereferenced)."""
+    ok = 1 << 20
+    d = _desc(k_pool=ok, v_pool=ok, node_parent=ok, node_kv_len=ok, node_page_offsets=ok, node_pages=ok,
+              path_leaf_node=ok, path_q_len=ok, q_offsets=ok, q=ok, out=ok + 16)
+    before = B.ss_launch_count()
+    ws = ctypes.c_void_p(1 << 21)
+    assert lib.ss_tree_attention(ctypes.byref(d), ws, ctypes.c_size_t(1 << 30), None) == B.SS_ERR_UNSUPPORTED
+    assert B.ss_launch_count() == before
+
+
 def test_dedup_and_topk_argument_validation_on_host(lib):
     null = ctypes.c_void_p(0)
     one = ctypes.c_void_p(256)     # never dereferenced: validation fails first

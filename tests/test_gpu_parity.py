@@ -5,6 +5,7 @@ Bars: dedup / remap / top-k bit-exact; attention |out - oracle| <= 2e-2 max and 
 would let through on long paths: dropping one 16-token page of a 4672-key path moves the output by only ~1.4e-3.
 """
 import math
+import os
 
 import numpy as np
 import pytest
@@ -20,6 +21,15 @@ DEV = "cuda:0"
 
 OUT_MAX, OUT_MEAN, LSE_MAX = 2e-2, 2e-3, 1e-3          # official
 TIGHT_OUT_MAX, TIGHT_OUT_MEAN, TIGHT_LSE = 6e-3, 4e-4, 2e-4   # internal, random N(0,1) data
+
+
+def log_observed(name, out_max, out_mean, lse_max):
+    """Appends the observed errors of one comparison to the file named by SS_PARITY_LOG (if set), so that the gates
+    below can be set from measurements."""
+    path = os.environ.get("SS_PARITY_LOG")
+    if path:
+        with open(path, "a") as f:
+            f.write(f"{name} out_max={out_max:.3e} out_mean={out_mean:.3e} lse_max={lse_max:.3e}\n")
 
 
 def check_dedup(r, w):
@@ -69,6 +79,7 @@ def check_attention(r, w, ref, max_paths=48, tight=True, host_w=None):
     fin = np.isfinite(l_ref)
     assert np.array_equal(np.isfinite(lse), fin)
     lerr = np.abs(lse[fin] - l_ref[fin]).max() if fin.any() else 0.0
+    log_observed(f"{w.name} tight={tight}", err.max(), err.mean(), lerr)
     assert err.max() <= OUT_MAX and err.mean() <= OUT_MEAN and lerr <= LSE_MAX, (err.max(), err.mean(), lerr)
     if tight:
         assert err.max() <= TIGHT_OUT_MAX and err.mean() <= TIGHT_OUT_MEAN and lerr <= TIGHT_LSE, \
@@ -426,12 +437,14 @@ def test_config5_full_size_sampled_outputs():
     lens = w.node_kv_len[w.path_leaf_node[uniq]]
     rng = np.random.default_rng(5)
     ver, dec = np.nonzero(T > 1)[0], np.nonzero(T == 1)[0]
-    pick = set(int(x) for x in rng.choice(ver, 14, replace=False)) | set(int(x) for x in rng.choice(dec, 40, replace=False))
+    # >= 128 unique paths: 44 verification paths (64 query tokens each) and 100 decode paths, plus the strata below
+    pick = set(int(x) for x in rng.choice(ver, 44, replace=False)) | set(int(x) for x in rng.choice(dec, 100, replace=False))
     pick |= {int(dec[lens[dec].argmin()]), int(dec[lens[dec].argmax()]), int(ver[lens[ver].argmin()]),
              int(ver[lens[ver].argmax()]), 0, U - 1}
     dup_u = np.nonzero(ref["multiplicity"] > 1)[0]
     pick |= {int(dup_u[0]), int(dup_u[-1])}
     sel = np.asarray(sorted(pick))
+    assert len(sel) >= 128 and (T[sel] > 1).sum() >= 40 and (T[sel] == 1).sum() >= 80
     sub = synth.extract_subworkload(w, uniq[sel])           # the needed pages and query rows, copied to the host
     o_ref, l_ref = oracle.tree_attention_workload(sub)
     off = np.concatenate([[0], np.cumsum(T.astype(np.int64))])
@@ -440,6 +453,7 @@ def test_config5_full_size_sampled_outputs():
     assert np.isfinite(out).all()
     err = np.abs(out - o_ref)
     lerr = np.abs(lse - l_ref).max()
+    log_observed("config5_full", err.max(), err.mean(), lerr)
     assert err.max() <= OUT_MAX and err.mean() <= OUT_MEAN and lerr <= LSE_MAX, (err.max(), err.mean(), lerr)
     assert err.max() <= TIGHT_OUT_MAX and err.mean() <= TIGHT_OUT_MEAN and lerr <= TIGHT_LSE, (err.max(), err.mean(), lerr)
 

@@ -54,6 +54,47 @@ def test_static_scratch_dedup_matches_workspace_dedup_twice_in_a_row():
             assert torch.equal(g, w)
 
 
+def test_static_scratch_dedup_small_and_empty_batches():
+    # batches of at most 4096 paths take the two-launch path, whose arrival counters live inside the shared scratch and
+    # must start at zero on every call; n = 0 writes only the count
+    for seed, n in [(3, 4096), (4, 300), (5, 1), (6, 4096)]:
+        ids, off, ctx, slot = _case(seed, n)
+        want = _run(False, ids, off, ctx, slot, n)
+        got = _run(True, ids, off, ctx, slot, n)
+        assert got[0] == want[0] and 0 < got[0] <= n
+        for g, w in zip(got[1:], want[1:]):
+            assert torch.equal(g, w)
+    one = torch.zeros(1, dtype=torch.int32, device=DEV)
+    off0 = torch.zeros(1, dtype=torch.int64, device=DEV)
+    outs = _outputs(1)
+    B.ss_dedup_paths_static(one, off0, None, None, 0, 0, outs[0], outs[1], outs[2], outs[3], None, outs[5])
+    torch.cuda.synchronize()
+    assert int(outs[5].item()) == 0
+    assert all(int(o.item()) == -5 for o in outs[:4])      # nothing but the count was written
+
+
+def test_static_scratch_dedup_at_its_maximum_and_without_allocating():
+    n = B.SS_DEDUP_STATIC_MAX_PATHS
+    ids, off, ctx, slot = _case(7, n)
+    want = _run(False, ids, off, ctx, slot, n)
+    got = _run(True, ids, off, ctx, slot, n)               # (also the warm call: the scratch address is now cached)
+    assert got[0] == want[0]
+    for g, w in zip(got[1:], want[1:]):
+        assert torch.equal(g, w)
+    # the property the entry point exists for: a call leaves the device's free memory and the framework's allocator
+    # exactly as it found them
+    canon, p2u, uniq, mult, slot_out, nu = _outputs(n)
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    alloc0, reserved0 = torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+    B.ss_dedup_paths_static(ids, off, ctx, slot, n, 0, canon, p2u, uniq, mult, slot_out, nu)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0
+    assert torch.cuda.memory_allocated() == alloc0 and torch.cuda.memory_reserved() == reserved0
+    assert int(nu.item()) == want[0]
+
+
 def test_static_scratch_dedup_rejects_batches_beyond_its_maximum():
     n = B.SS_DEDUP_STATIC_MAX_PATHS + 1
     one = torch.zeros(1, dtype=torch.int32, device=DEV)
