@@ -176,6 +176,188 @@ def time_oracle(w_host, steps, warmup):
 
 
 # ------------------------------------------------------------------------------------------------------------
+# the smaller benchmark configurations and the "next" rows, reported inside the default run's JSON line
+# ------------------------------------------------------------------------------------------------------------
+def timed_ms(fn, steps, flush, dev):
+    """CUDA-event time of `fn` per call, `steps` calls, L2 evicted before each (outside the events)."""
+    import torch
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for i, (a, b) in enumerate(ev):
+        if flush is not None:
+            flush.fill_(i & 0xff)
+        a.record()
+        fn()
+        b.record()
+    torch.cuda.synchronize(dev)
+    return [a.elapsed_time(b) for a, b in ev]
+
+
+def small_workload(name, dev, flush, peaks, steps=20, warmup=5):
+    """One of c2 / c3 / c4 (each well under a millisecond per step): whole step, attention call alone, per-phase
+    times (the library's event profiler) and the two roofline fractions, with the clocks sampled meanwhile."""
+    import torch
+    from paper_2609_39334_b200 import binding as B
+    from paper_2609_39334_b200 import synth
+    from paper_2609_39334_b200.pipeline import DevicePipeline
+    w = synth.make_config(WORKLOADS[name], device=dev, poison=True)
+    pipe = DevicePipeline(w, dev)
+    for _ in range(warmup):
+        pipe.step()
+    torch.cuda.synchronize(dev)
+    st = B.ss_last_device_status(pipe.attn_ws)
+    if st != B.SS_OK:
+        raise B.SpecScaleError(st, f"{name} warm-up")
+    clocks = ClockSampler(dev.index or 0)
+    clocks.start()
+    time.sleep(0.12)
+    launches0 = B.ss_launch_count()
+    step_ms = timed_ms(pipe.step, steps, flush, dev)
+    launches = (B.ss_launch_count() - launches0) // steps
+    attn_ms = timed_ms(pipe.attention, steps, flush, dev)
+    B.ss_profile_read()
+    B.ss_profile_enable(True)
+    timed_ms(pipe.attention, steps, flush, dev)
+    B.ss_profile_enable(False)
+    phase_ms, phase_calls = B.ss_profile_read()
+    time.sleep(0.12)
+    clk = clocks.stop()
+    st = B.ss_last_device_status(pipe.attn_ws)
+    if st != B.SS_OK:
+        raise B.SpecScaleError(st, name)
+    U = int(pipe.num_unique.item())
+    work = algorithmic_work(w, pipe.unique_paths[:U].cpu().numpy())
+    tokens = work["tokens"]
+    phases = {k: (phase_ms[k] / phase_calls[k] if phase_calls[k] else 0.0) for k in phase_ms}
+    out = {"paths": w.num_paths, "unique_paths": U, "query_tokens": tokens,
+           "heads": f"{w.num_q_heads}q/{w.num_kv_heads}kv", "launches_per_step": int(launches),
+           "step_ms_median": float(np.median(step_ms)), "step_ms_min": float(min(step_ms)),
+           "tokens_per_s": tokens / (float(np.median(step_ms)) * 1e-3),
+           "attention_ms_median": float(np.median(attn_ms)), "attention_ms_min": float(min(attn_ms)),
+           "attention_tokens_per_s": tokens / (float(np.median(attn_ms)) * 1e-3),
+           "phase_ms": phases,
+           "phase_note": "phase times carry the profiler's events (a few microseconds each); the attention and step "
+                         "times above are measured without them",
+           "l2": "L2 flushed between iterations", "steps": steps, "warmup": warmup, "clocks": clk}
+    if phases.get("tiles"):
+        ach = work["tile_flops"] / (phases["tiles"] * 1e-3) / 1e12
+        out["tiles"] = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_burst"], "unit": "TFLOP/s",
+                        "frac": ach / peaks["bf16_burst"], "peak_kind": f"{peaks['source']} burst"}
+    if phases.get("leaves") and work["leaf_bytes"] > 0:
+        ach = work["leaf_bytes"] / (phases["leaves"] * 1e-3) / 1e9
+        out["leaves"] = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": ach / peaks["hbm_gbs"], "peak_kind": f"{peaks['source']} copy",
+                         "note": "the leaf launch also merges the partial results and writes the final rows"}
+    hbm_s = work["unique_kv_bytes"] / (peaks["hbm_gbs"] * 1e9)
+    tensor_s = work["tile_flops"] / (peaks["bf16_burst"] * 1e12)
+    out["attention_roofline_ms"] = 1e3 * max(hbm_s, tensor_s)
+    out["attention_frac_of_roofline"] = out["attention_roofline_ms"] / out["attention_ms_median"]
+    del pipe, w
+    torch.cuda.empty_cache()
+    return out
+
+
+def next_rows(dev, flush, peaks, steps=20):
+    """Numbers for the rows beyond the core path: on-demand branching draws, radix-tree construction, early pruning
+    with partially verified candidates, and the knee of the verification-batch curve."""
+    import torch
+    from paper_2609_39334_b200 import binding as B
+    rng = np.random.default_rng(12345)
+    out = {}
+    # ---- ss_branch_sample: c2-shaped expansion (922 sequences drawing ~1024 candidates from 151936-token rows) --------
+    S, V = 922, 151936
+    logits = torch.randn((S, V), dtype=torch.float32, device=dev) * 3
+    pot = rng.integers(1, 3, size=S)
+    off = torch.from_numpy(np.concatenate([[0], np.cumsum(pot)]).astype(np.int64)).to(dev)
+    n = int(pot.sum())
+    u = torch.from_numpy(rng.random(n).astype(np.float32)).to(dev)
+    tok = torch.empty(n, dtype=torch.int32, device=dev)
+    seq = torch.empty(n, dtype=torch.int64, device=dev)
+    fn = lambda: B.ss_branch_sample(logits, off, u, S, V, 0.8, tok, seq)
+    fn()
+    ms = float(np.median(timed_ms(fn, steps, flush, dev)))
+    gbs = S * V * 4 / (ms * 1e-3) / 1e9
+    out["ss_branch_sample"] = {"sequences": S, "vocab": V, "draws": n, "ms": ms, "logit_gb_per_s": gbs,
+                               "frac_of_hbm": gbs / peaks["hbm_gbs"], "algorithmic_bytes": "4 B per logit, read once"}
+    del logits
+    # ---- ss_build_prefix_tree: c5-shaped ids (64 prompts of 4096 tokens x 256 candidates with 128-1024 own tokens) ----
+    P_, F_ = 64, 256
+    lens = rng.integers(128, 1025, size=P_ * F_) + 4096
+    off_np = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    total = int(off_np[-1])
+    ids = torch.randint(0, 151936, (total,), dtype=torch.int32, device=dev)
+    off_t = torch.from_numpy(off_np).to(dev)
+    prompts = torch.randint(0, 151936, (P_, 4096), dtype=torch.int32, device=dev)
+    starts = off_t[:-1]
+    idx = (starts[:, None] + torch.arange(4096, device=dev)[None, :]).reshape(-1)
+    ids[idx] = prompts.repeat_interleave(F_, dim=0).reshape(-1)
+    del idx, prompts
+    npaths = P_ * F_
+    i32 = dict(dtype=torch.int32, device=dev)
+    order, leaf = torch.empty(npaths, **i32), torch.empty(npaths, **i32)
+    parent, kv, sp, so = (torch.empty(2 * npaths, **i32) for _ in range(4))
+    num = torch.zeros(1, **i32)
+    ws = B.alloc_workspace(B.ss_prefix_tree_workspace_bytes(npaths, total, 16), dev)
+    fn = lambda: B.ss_build_prefix_tree(ids, off_t, npaths, total, 16, order, leaf, parent, kv, sp, so, num, ws)
+    fn()
+    ms = float(np.median(timed_ms(fn, max(steps // 4, 3), None, dev)))
+    out["ss_build_prefix_tree"] = {"paths": npaths, "token_ids": total, "nodes": int(num.item()), "ms": ms,
+                                   "id_gb_per_s": total * 4 / (ms * 1e-3) / 1e9,
+                                   "status": B.ss_last_device_status(ws)}
+    del ids, ws
+    # ---- ss_early_prune: c5-shaped segments (64 problems x 256 candidates, half of them verified, k = 64) ----------------
+    n = 16384
+    scores = torch.from_numpy(np.round(rng.random(n) * 8).astype(np.float32) / 8).to(dev)
+    verified = torch.from_numpy((rng.random(n) < 0.5).astype(np.uint8)).to(dev)
+    seg = torch.arange(0, n + 1, 256, dtype=torch.int32, device=dev)
+    pruned = torch.empty(n, dtype=torch.uint8, device=dev)
+    selected = torch.empty((64, 64), **i32)
+    final = torch.empty(64, dtype=torch.uint8, device=dev)
+    ws = B.alloc_workspace(B.ss_topk_workspace_bytes(n), dev)
+    fn = lambda: B.ss_early_prune(scores, verified, seg, 64, n, 64, pruned, selected, final, ws)
+    fn()
+    out["ss_early_prune"] = {"candidates": n, "segments": 64, "k": 64,
+                             "ms": float(np.median(timed_ms(fn, steps, flush, dev)))}
+    torch.cuda.empty_cache()
+    return out
+
+
+def lv_curve(dev, flush, steps, warmup):
+    """Verification-attention throughput against the number of batched step tokens (see lv_sweep)."""
+    import torch
+    from paper_2609_39334_b200 import binding as B
+    from paper_2609_39334_b200 import synth
+    from paper_2609_39334_b200.pipeline import DevicePipeline
+    curve = []
+    for target in LV_SWEEP_TOKENS:
+        problems = max(1, target // (8 * 72))
+        per = max(1, round(target / (72 * problems)))
+        w = synth.build_tree_workload(f"lv{target}", synth.BASE_SEED + 100 + target, 28, 4, [1024], [per], problems,
+                                      (64, 512), lambda i, n, rng: int(rng.integers(16, 129)), device=dev)
+        pipe = DevicePipeline(w, dev)
+        pipe.dedup()
+        pipe.compact_unique()
+        for _ in range(max(warmup, 3)):
+            pipe.attention()
+        torch.cuda.synchronize(dev)
+        ms = float(np.median(timed_ms(pipe.attention, steps, flush, dev)))
+        st = B.ss_last_device_status(pipe.attn_ws)
+        if st != B.SS_OK:
+            raise B.SpecScaleError(st, "lv-sweep")
+        tokens = int(w.path_q_len.sum())
+        curve.append({"batched_tokens": tokens, "candidates": w.num_paths, "ms": ms, "tokens_per_s": tokens / (ms * 1e-3)})
+        del pipe, w
+    # knee: the smallest batch that reaches 90 % of the largest batch's tokens/s (linear interpolation between points)
+    top = curve[-1]["tokens_per_s"]
+    knee = None
+    for a, b in zip(curve, curve[1:]):
+        if a["tokens_per_s"] < 0.9 * top <= b["tokens_per_s"]:
+            f = (0.9 * top - a["tokens_per_s"]) / (b["tokens_per_s"] - a["tokens_per_s"])
+            knee = a["batched_tokens"] + f * (b["batched_tokens"] - a["batched_tokens"])
+    if knee is None and curve[0]["tokens_per_s"] >= 0.9 * top:
+        knee = curve[0]["batched_tokens"]
+    return curve, knee
+
+
 def lv_sweep(args):
     """Attention-only analogue of the paper's verification-throughput profile (Section "Lazy Verification": the
     token threshold of the first flush policy is read off a throughput-vs-batched-tokens curve).  For each batch
@@ -191,35 +373,13 @@ def lv_sweep(args):
     if int(os.environ.get("RANK", "0")) != 0:
         return
     flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=dev)
-    curve = []
-    for target in LV_SWEEP_TOKENS:
-        problems = max(1, target // (8 * 72))
-        per = max(1, round(target / (72 * problems)))
-        w = synth.build_tree_workload(f"lv{target}", synth.BASE_SEED + 100 + target, 28, 4, [1024], [per], problems,
-                                      (64, 512), lambda i, n, rng: int(rng.integers(16, 129)), device=dev)
-        pipe = DevicePipeline(w, dev)
-        pipe.dedup()
-        pipe.compact_unique()
-        for _ in range(max(args.warmup, 3)):
-            pipe.attention()
-        torch.cuda.synchronize(dev)
-        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-        for a, b in ev:
-            flush.fill_(1)
-            a.record()
-            pipe.attention()
-            b.record()
-        torch.cuda.synchronize(dev)
-        st = B.ss_last_device_status(pipe.attn_ws)
-        if st != B.SS_OK:
-            raise B.SpecScaleError(st, "lv-sweep")
-        ms = float(np.median([a.elapsed_time(b) for a, b in ev]))
-        tokens = int(w.path_q_len.sum())
-        curve.append({"batched_tokens": tokens, "candidates": w.num_paths, "ms": ms, "tokens_per_s": tokens / (ms * 1e-3)})
+    curve, knee = lv_curve(dev, flush, args.steps, args.warmup)
     print(json.dumps({"metric": "verification_attention_step_tokens_per_s", "unit": "tokens/s", "n_gpus": 1,
                       "steps": args.steps, "warmup": max(args.warmup, 3), "dtype": "bf16", "data": "synthetic",
                       "config": {"workload": "lv-sweep", "heads": "28q/4kv", "prefix": 1024, "l2": "L2 flushed between iterations"},
-                      "curve": curve}))
+                      "curve": curve, "knee_tokens_at_90pct": knee,
+                      "paper_context": "the paper's reward-model forward saturates near 2048 batched tokens on an A100 "
+                                       "(Section Lazy Verification); this curve is the attention call alone on a B200"}))
 
 
 def main():
@@ -233,12 +393,15 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--tiles-2cta", action="store_true",
                     help="run the tile items on the two-CTAs-per-SM kernel (64-key tiles) instead of the default one")
+    ap.add_argument("--tiles-flow", action="store_true", help="run the tile items on the free-running kernel")
     ap.add_argument("--graph", action="store_true",
                     help="also time the step as a CUDA graph replay (reported as ms_per_step_cuda_graph)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-depth", type=int, default=3,
                     help="independent (host buffers, device arena, stream) sets the end-to-end leg alternates between")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-workloads", action="store_true",
+                    help="skip the c2 / c3 / c4 and next-row measurements that the default run appends (`workloads`, `next_rows`)")
     ap.add_argument("--profiler-range", action="store_true",
                     help="bracket the timed region with cudaProfilerStart/Stop (for ncu --profile-from-start off)")
     args = ap.parse_args()
@@ -299,7 +462,7 @@ def main():
     # every rank its own problems: same shapes, different seed
     from paper_2609_39334_b200 import replicas
     w = replicas.replica_workload(synth.make_config, cfg_idx, rank, device=dev, scale=args.scale, poison=True)
-    pipe = DevicePipeline(w, dev, attn_flags=B.SS_FLAG_TILES_2CTA if args.tiles_2cta else 0)
+    pipe = DevicePipeline(w, dev, attn_flags=B.SS_FLAG_TILES_2CTA if args.tiles_2cta else (B.SS_FLAG_TILES_FLOW if args.tiles_flow else 0))
     kv_bytes = pipe.kv_pool.numel() * 2
     flush = None
     if kv_bytes < 4 * L2_BYTES:
@@ -490,6 +653,20 @@ def main():
             "value": stok / sec, "unit": UNIT, "cores": oracle.host_cores(), "kind": "oracle",
             "sample": f"{len(sample)} unique paths of {args.workload} ({int((sub.path_q_len > 1).sum())} verification, "
                       f"{int((sub.path_q_len == 1).sum())} decode), {stok} query tokens, {sec:.1f} s"}
+
+    # ---- the other benchmark configurations and the rows beyond the core path (default run, rank 0, N = 1) ------------
+    if rank == 0 and world == 1 and args.workload == "c5" and args.scale == 1.0 and not args.no_workloads:
+        del pipe
+        w.kv_pool = None
+        w.q = None
+        torch.cuda.empty_cache()
+        small_flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=dev)
+        out["workloads"] = {name: small_workload(name, dev, small_flush, peaks) for name in ("c2", "c3", "c4")}
+        out["next_rows"] = next_rows(dev, small_flush, peaks)
+        curve, knee = lv_curve(dev, small_flush, 20, 3)
+        out["next_rows"]["lv_sweep"] = {"curve": curve, "knee_tokens_at_90pct": knee,
+                                        "paper_context": "reward-model forward saturates near 2048 batched tokens on an A100"}
+        del small_flush
 
     if rank == 0:
         print(json.dumps(out))

@@ -54,6 +54,8 @@ extern "C" {
 #define SS_FLAG_TILES_2CTA 0x10u    /* attention: run the tcgen05 tile items on the kernel that keeps two CTAs
                                        per SM and works on 64-key tiles (default: the one-CTA-per-SM kernel with
                                        128-key tiles); same results within the accuracy contract             */
+#define SS_FLAG_TILES_FLOW 0x20u    /* attention: run the tcgen05 tile items on the free-running kernel (roles do
+                                       not meet at item ends, two accumulators); same results                 */
 
 #define SS_MAX_DEPTH 16             /* maximum number of nodes on a root-to-leaf chain                       */
 

@@ -13,7 +13,9 @@ from typing import Optional
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libspecscale.so")
+# SS_LIB_SUFFIX selects a build variant (build.build(defines=..., suffix=...)): "_checked" for the build with device-side
+# range checks, or an instrumented build; the default is the production library.
+LIB_PATH = os.path.join(_HERE, "libspecscale" + os.environ.get("SS_LIB_SUFFIX", "") + ".so")
 
 SS_OK = 0
 SS_ERR_INVALID_ARG = 1
@@ -27,6 +29,7 @@ SS_FLAG_FORCE_GENERIC = 0x2
 SS_FLAG_NO_TCGEN05 = 0x4
 SS_FLAG_WEAK_HASH = 0x8
 SS_FLAG_TILES_2CTA = 0x10
+SS_FLAG_TILES_FLOW = 0x20
 SS_MAX_DEPTH = 16
 SS_DEDUP_STATIC_MAX_PATHS = 65536
 

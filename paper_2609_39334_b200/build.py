@@ -24,26 +24,30 @@ def sources():
     return sorted(glob.glob(os.path.join(CSRC, "*.cu")))
 
 
-def _stale() -> bool:
-    if not os.path.exists(LIB):
+def _stale(lib: str = LIB) -> bool:
+    if not os.path.exists(lib):
         return True
-    t = os.path.getmtime(LIB)
+    t = os.path.getmtime(lib)
     deps = sources() + glob.glob(os.path.join(CSRC, "*.cuh")) + \
         glob.glob(os.path.join(_HERE, "..", "include", "*.h"))
     return any(os.path.getmtime(f) > t for f in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and not _stale():
-        return LIB
-    objdir = os.path.join(_HERE, "build")
+def build(force: bool = False, verbose: bool = False, defines=(), suffix: str = "") -> str:
+    """Builds libspecscale<suffix>.so.  `defines` are extra -D macros (an instrumented or checked variant gets its own
+    suffix and object directory); SS_NVCC_DEFINES in the environment adds more, comma separated."""
+    defines = list(defines) + [d for d in os.environ.get("SS_NVCC_DEFINES", "").split(",") if d]
+    lib = LIB[:-3] + suffix + ".so"
+    if not force and not _stale(lib):
+        return lib
+    objdir = os.path.join(_HERE, "build" + suffix)
     os.makedirs(objdir, exist_ok=True)
     procs = []
     objs = []
     for src in sources():
         obj = os.path.join(objdir, os.path.basename(src)[:-3] + ".o")
         objs.append(obj)
-        cmd = [NVCC, *FLAGS, *FILE_FLAGS.get(os.path.basename(src), []), "-c", src, "-o", obj]
+        cmd = [NVCC, *FLAGS, *[f"-D{d}" for d in defines], *FILE_FLAGS.get(os.path.basename(src), []), "-c", src, "-o", obj]
         if verbose:
             cmd.insert(1, "-Xptxas")
             cmd.insert(2, "-v")
@@ -56,10 +60,10 @@ def build(force: bool = False, verbose: bool = False) -> str:
         failed |= p.returncode != 0
     if failed:
         raise RuntimeError("nvcc failed")
-    tmp = LIB + f".tmp{os.getpid()}"
+    tmp = lib + f".tmp{os.getpid()}"
     subprocess.check_call([NVCC, "-shared", "-o", tmp, *objs, "-Xcompiler", "-fPIC"])
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":

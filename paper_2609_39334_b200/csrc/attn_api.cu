@@ -16,6 +16,9 @@ int32_t launch_merge(const Params& P, cudaStream_t st, int sm_count);
 int32_t launch_leaf_items(const Params& P, cudaStream_t st, int sm_count);
 int32_t launch_tile_items_umma(const Params& P, cudaStream_t st, int sm_count);
 int32_t launch_tile_items_umma_split(const Params& P, cudaStream_t st, int sm_count);
+int32_t launch_tile_items_umma_flow(const Params& P, cudaStream_t st, int sm_count);
+bool leaf_stream_supported(const Params& P);
+int32_t launch_leaf_stream(const Params& P, cudaStream_t st, int sm_count);
 
 // ---- per-phase event timing (diagnostics) ------------------------------------------------------------------
 constexpr int kProfCalls = 256;                      // timed calls between two reads
@@ -58,7 +61,7 @@ static int sm_count_of_current_device() {
 
 static int32_t check_desc(const ss_attn_desc_t* d) {
   if (!d || d->struct_size != sizeof(ss_attn_desc_t)) return SS_ERR_INVALID_ARG;
-  if (d->flags & ~(SS_FLAG_VALIDATE | SS_FLAG_FORCE_GENERIC | SS_FLAG_NO_TCGEN05 | SS_FLAG_TILES_2CTA)) return SS_ERR_INVALID_ARG;
+  if (d->flags & ~(SS_FLAG_VALIDATE | SS_FLAG_FORCE_GENERIC | SS_FLAG_NO_TCGEN05 | SS_FLAG_TILES_2CTA | SS_FLAG_TILES_FLOW)) return SS_ERR_INVALID_ARG;
   if (d->num_q_heads < 1 || d->num_kv_heads < 1 || d->num_nodes < 0 || d->num_paths < 0 || d->total_q < 0 ||
       d->total_node_pages < 0 || d->num_pages < 0 || d->max_depth < 0 || d->max_decode_paths < 0)
     return SS_ERR_INVALID_ARG;
@@ -86,13 +89,20 @@ static Layout carve(const ss_attn_desc_t* d, char* base, Params* P) {
   const int64_t cap_dec = d->max_decode_paths > 0 ? (d->max_decode_paths < d->num_paths ? d->max_decode_paths : d->num_paths)
                                                   : d->num_paths;
   const int target = 2 * sm_count_of_current_device();   // (the size query and the call must see the same device)
+  // Keys per leaf item.  The leaf kernel runs ~12 warps per SM, each a pipeline of its own; with fewer than about eight
+  // items per warp the longest warp sets the kernel's time, so small calls cut the leaves finer (more partials to
+  // merge, which stay in L2).  Decided from host-side numbers only, so that the capacities below match the plan.
+  const int64_t page_items = d->total_node_pages * Hkv;
+  const int64_t warp_slots = 12LL * sm_count_of_current_device();
+  (void)page_items; (void)warp_slots;
+  const int leaf_chunk = kLeafChunk;
   Caps caps;
   caps.dec = static_cast<int32_t>(cap_dec);
   const int64_t stacked = static_cast<int64_t>(Hkv) * (cap_dec * max_depth / tpt + d->num_nodes) + target + Hkv * kMaxRootSplits;
   const int64_t chain = static_cast<int64_t>(Hkv) * (d->total_q / tpt + d->num_paths);
   caps.tile_items = static_cast<int32_t>(stacked + chain);
-  caps.leaf_items = static_cast<int32_t>(static_cast<int64_t>(Hkv) * (d->total_node_pages * kPage / kLeafChunk + cap_dec));
-  caps.slots = cap_dec * (kMaxRootSplits + max_depth) + d->total_node_pages * kPage / kLeafChunk;
+  caps.leaf_items = static_cast<int32_t>(static_cast<int64_t>(Hkv) * (d->total_node_pages * kPage / leaf_chunk + cap_dec));
+  caps.slots = cap_dec * (kMaxRootSplits + max_depth) + d->total_node_pages * kPage / leaf_chunk;
 
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return base ? base + o : nullptr; };
@@ -105,6 +115,8 @@ static Layout carve(const ss_attn_desc_t* d, char* base, Params* P) {
   char* dec_tok = take((static_cast<size_t>(cap_dec) + 1) * 4);
   char* dec_src = take((static_cast<size_t>(cap_dec) + 1) * 4);
   char* dec_slot = take((static_cast<size_t>(cap_dec) + 1) * 4);
+  char* dec_chunks = take((static_cast<size_t>(cap_dec) + 1) * 4);
+  char* leaf_arrive = take((static_cast<size_t>(cap_dec) * Hkv + 1) * 4);
   char* tiles = take(static_cast<size_t>(caps.tile_items) * sizeof(TileItem));
   char* leaves = take(static_cast<size_t>(caps.leaf_items) * sizeof(LeafItem));
   char* part_o = take(static_cast<size_t>(caps.slots) * d->num_q_heads * kHeadDim * 4);
@@ -120,12 +132,15 @@ static Layout carve(const ss_attn_desc_t* d, char* base, Params* P) {
     P->dec_tok = reinterpret_cast<int32_t*>(dec_tok);
     P->dec_src = reinterpret_cast<int32_t*>(dec_src);
     P->dec_slot_base = reinterpret_cast<int32_t*>(dec_slot);
+    P->dec_leaf_chunks = reinterpret_cast<int32_t*>(dec_chunks);
+    P->leaf_arrive = reinterpret_cast<int32_t*>(leaf_arrive);
     P->tile_items = reinterpret_cast<TileItem*>(tiles);
     P->leaf_items = reinterpret_cast<LeafItem*>(leaves);
     P->part_o = reinterpret_cast<float*>(part_o);
     P->part_lse = reinterpret_cast<float*>(part_lse);
     P->caps = caps;
     P->target_tiles = target;
+    P->leaf_chunk = leaf_chunk;
   }
   Layout L;
   L.total = off;
@@ -159,6 +174,7 @@ extern "C" int32_t ss_tree_attention(const ss_attn_desc_t* d, void* workspace, s
       reinterpret_cast<uintptr_t>(d->q) % 16 || reinterpret_cast<uintptr_t>(d->out) % 32)
     return SS_ERR_UNSUPPORTED;
   if (d->total_q > 0x7fffffffLL / d->num_q_heads) return SS_ERR_UNSUPPORTED;   // row indices are int32
+  if (d->total_node_pages > 0x7fffffffLL) return SS_ERR_UNSUPPORTED;           // so are indices into node_pages
   if (d->q_src_offsets && (d->q_src_rows < 0 || d->q_src_rows > 0x7fffffffLL / d->num_q_heads)) return SS_ERR_INVALID_ARG;
 
   Params P;
@@ -212,22 +228,27 @@ extern "C" int32_t ss_tree_attention(const ss_attn_desc_t* d, void* workspace, s
   if (rc == SS_OK && any && !generic_only) {
     const bool two_cta = (d->flags & SS_FLAG_TILES_2CTA) != 0;
     rc = simple ? launch_tile_items_simple(P, st, sms)
-                : (two_cta ? launch_tile_items_umma(P, st, sms) : launch_tile_items_umma_split(P, st, sms));
+                : (two_cta ? launch_tile_items_umma(P, st, sms)
+                           : ((d->flags & SS_FLAG_TILES_FLOW) ? launch_tile_items_umma_flow(P, st, sms)
+                                                              : launch_tile_items_umma_split(P, st, sms)));
     ran(SS_PHASE_TILES);
   }
+  // Decode leaves.  The streaming kernel also merges the per-level partials and computes the rows of GENERIC paths;
+  // pools it cannot take (and the plain mode) go through the register-staged leaf kernel and a merge launch.
+  const bool fused_finish = !simple && !generic_only && leaf_stream_supported(P);
   mark(SS_PHASE_LEAVES);
   if (rc == SS_OK && any && !generic_only) {
-    rc = simple ? launch_leaf_items_simple(P, st, sms) : launch_leaf_items(P, st, sms);
+    rc = simple ? launch_leaf_items_simple(P, st, sms) : (fused_finish ? launch_leaf_stream(P, st, sms) : launch_leaf_items(P, st, sms));
     ran(SS_PHASE_LEAVES);
   }
   mark(SS_PHASE_GENERIC);
-  if (rc == SS_OK && any) {
+  if (rc == SS_OK && any && generic_only) {
     rc = launch_generic(P, st, sms);
     ran(SS_PHASE_GENERIC);
   }
   mark(SS_PHASE_MERGE);
-  if (rc == SS_OK && any && !generic_only) {
-    rc = launch_merge(P, st, sms);
+  if (rc == SS_OK && any && !generic_only && !fused_finish) {
+    rc = launch_merge(P, st, sms);                    // (rows of GENERIC paths, then the merge)
     ran(SS_PHASE_MERGE);
   }
   mark(SS_NUM_PHASES);

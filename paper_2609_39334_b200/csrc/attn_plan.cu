@@ -1,12 +1,18 @@
 // Device-side planner of ss_tree_attention: turns the tree + per-path arrays into work lists (tile items, leaf
 // items), partial-slot assignments and per-path classes.  Running it on the device means the live path count can
-// come straight from ss_dedup_paths without a host round trip.  Four small launches on the caller's stream:
-//   plan_nodes   (grid over nodes)   depth and prefix length of every node, range checks, counters reset
-//   plan_paths   (grid over paths)   class and key length of every path, membership counts of its chain nodes
-//   plan_scan    (one block)         every prefix sum: decode ranks, per-node tile items and KV splits, partial
-//                                    slots, leaf items, chain items; capacity checks; totals into the header
-//   plan_emit    (grid)              writes the item lists and the per-decode-token arrays
-// The header (status word first) is cleared by the host-side launcher before plan_nodes.
+// come straight from ss_dedup_paths without a host round trip.  Four phases:
+//   nodes   depth and prefix length of every node, range checks, counters reset
+//   paths   class and key length of every path, membership counts of its chain nodes
+//   scan    (one block) every prefix sum: decode ranks, per-node tile items and KV splits, partial slots, leaf
+//           items, chain items; capacity checks; totals into the header
+//   emit    writes the item lists and the per-decode-token arrays
+// Trees of up to kSmallPlan nodes and paths (every benchmark configuration but the largest) are planned by ONE
+// block in ONE launch: the tree arrays and all intermediate arrays live in shared memory (the phase functions only
+// see redirected pointers), so the whole plan costs three or four round trips to global memory instead of the
+// dozens that the dependent loads and in-place scans of the general path make.  Larger inputs take four launches
+// (nodes, paths and emit grid-parallel, scan in one block).
+// The header (status word first) is cleared by the host-side launcher before the first of the four kernels; the
+// one-block planner builds it in shared memory and writes it out whole.
 #include "attn_plan.cuh"
 
 namespace ss {
@@ -76,8 +82,7 @@ __device__ __forceinline__ int live_paths(const Params& P) {
 }
 
 // ---- nodes: depth and number of keys before the node -------------------------------------------------------------
-__global__ void __launch_bounds__(kGridThreads) plan_nodes_kernel(const Params P) {
-  ss::grid_dependency_enter();
+__device__ __forceinline__ void plan_nodes_phase(const Params& P) {
   PlanHeader* hdr = P.hdr;
   const int64_t gtid = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   const int64_t gsize = static_cast<int64_t>(gridDim.x) * blockDim.x;
@@ -116,11 +121,9 @@ __global__ void __launch_bounds__(kGridThreads) plan_nodes_kernel(const Params P
 }
 
 // ---- paths: class, kv length, membership counts of every chain node ------------------------------------------------
-__global__ void __launch_bounds__(kGridThreads) plan_paths_kernel(const Params P) {
-  ss::grid_dependency_enter();
+__device__ __forceinline__ void plan_paths_phase(const Params& P) {
   PlanHeader* hdr = P.hdr;
-  if (hdr->status != SS_OK) return;          // no barrier in this kernel: a per-thread return is safe
-  const int live = hdr->live_paths;
+  const int live = live_paths(P);
   const int N = P.num_nodes;
   const bool force_generic = (P.flags & SS_FLAG_FORCE_GENERIC) != 0;
   const int64_t gsize = static_cast<int64_t>(gridDim.x) * blockDim.x;
@@ -159,13 +162,12 @@ __global__ void __launch_bounds__(kGridThreads) plan_paths_kernel(const Params P
 }
 
 // ---- every prefix sum -------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kScanThreads) plan_scan_kernel(const Params P) {
-  ss::grid_dependency_enter();
+__device__ __forceinline__ void plan_scan_phase(const Params& P) {   // one whole block; block-uniform returns only
   __shared__ int s_total_tiles;
   PlanHeader* hdr = P.hdr;
   if (block_failed(hdr)) return;
   const int tid = threadIdx.x, nt = blockDim.x;
-  const int live = hdr->live_paths;
+  const int live = live_paths(P);
   const int N = P.num_nodes;
   const int tpt = P.tok_per_tile;
   if (tid == 0) s_total_tiles = 0;
@@ -200,7 +202,7 @@ __global__ void __launch_bounds__(kScanThreads) plan_scan_kernel(const Params P)
     int splits = 1, own = 0, split_len = len;
     if (nd > 0 && len > 0) {
       if (tiles == 0) {
-        own = ceil_div(len, kLeafChunk);             // private leaf of one decode path
+        own = ceil_div(len, P.leaf_chunk);             // private leaf of one decode path
       } else {
         if (P.node_depth[n] == 0 && total_tiles < P.target_tiles) {
           int want = ceil_div(P.target_tiles, total_tiles);
@@ -237,7 +239,7 @@ __global__ void __launch_bounds__(kScanThreads) plan_scan_kernel(const Params P)
       const int leaf = P.path_leaf_node[p];
       slots = P.node_level_off[leaf] + P.node_own_slots[leaf];
       if (P.node_npaths[leaf] == 1 && P.node_kv_len[leaf] > 0)
-        leaf_items = ceil_div(P.node_kv_len[leaf], kLeafChunk) * P.Hkv;
+        leaf_items = ceil_div(P.node_kv_len[leaf], P.leaf_chunk) * P.Hkv;
     } else if (cls == kClassChain) {
       chain_items = ceil_div(P.path_q_len[p], tpt) * P.Hkv;
     }
@@ -261,11 +263,9 @@ __global__ void __launch_bounds__(kScanThreads) plan_scan_kernel(const Params P)
 }
 
 // ---- item lists ---------------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kGridThreads) plan_emit_kernel(const Params P) {
-  ss::grid_dependency_enter();
+__device__ __forceinline__ void plan_emit_phase(const Params& P) {
   PlanHeader* hdr = P.hdr;
-  if (hdr->status != SS_OK) return;          // no barrier in this kernel
-  const int live = hdr->live_paths;
+  const int live = live_paths(P);
   const int N = P.num_nodes;
   const int tpt = P.tok_per_tile;
   const int n_stacked = hdr->n_stacked_items;
@@ -273,56 +273,91 @@ __global__ void __launch_bounds__(kGridThreads) plan_emit_kernel(const Params P)
   const int64_t gsize = static_cast<int64_t>(gridDim.x) * blockDim.x;
   if (gtid == 0) P.dec_slot_base[hdr->n_dec] = hdr->n_slots;
 
+  // per decode token: output row, query row, partial slots, leaf chunks, arrival counters
   for (int64_t p64 = gtid; p64 < live; p64 += gsize) {
     const int p = static_cast<int>(p64);
-    const int cls = P.path_class[p];
-    if (cls == kClassDecode) {
-      const int rank = P.path_dec_rank[p];
-      const int leaf = P.path_leaf_node[p];
-      const int len = P.node_kv_len[leaf];
-      const int32_t src_row = static_cast<int32_t>(P.q_src_offsets ? P.q_src_offsets[p] : P.q_offsets[p]);
-      P.dec_tok[rank] = static_cast<int32_t>(P.q_offsets[p]);
-      P.dec_src[rank] = src_row;
-      P.dec_slot_base[rank] = P.path_slot_base[p];
-      if (!(P.node_npaths[leaf] == 1 && len > 0)) continue;
-      const int chunks = ceil_div(len, kLeafChunk);
-      int e = P.path_leaf_base[p];
-      const int slot0 = P.path_slot_base[p] + P.node_level_off[leaf];
-      for (int c = 0; c < chunks; ++c)
-        for (int g = 0; g < P.Hkv; ++g) {
-          LeafItem it;
-          it.q_row = static_cast<int32_t>(P.q_offsets[p]);
-          it.node = leaf;
-          it.g = g;
-          it.kv_begin = c * kLeafChunk;
-          it.kv_end = min(len, (c + 1) * kLeafChunk);
-          it.slot = slot0 + c;
-          it.q_src = src_row;
-          it.pad1 = 0;
-          P.leaf_items[e++] = it;
-        }
-    } else if (cls == kClassChain) {
-      const int T = P.path_q_len[p];
-      const int L = P.path_kv_len[p];
-      const int tiles = ceil_div(T, tpt);
-      const int32_t src_row = static_cast<int32_t>(P.q_src_offsets ? P.q_src_offsets[p] : P.q_offsets[p]);
-      int e = n_stacked + P.path_chain_base[p];
-      for (int g = 0; g < P.Hkv; ++g)
-        for (int t = 0; t < tiles; ++t) {
-          TileItem it;
-          it.node = P.path_leaf_node[p];
-          it.tok0 = static_cast<int32_t>(P.q_offsets[p]) + t * tpt;
-          it.n_tok = min(tpt, T - t * tpt);
-          it.kind_g = (kItemChain << 16) | g;
-          it.kv_begin = 0;
-          it.limit0 = L - T + t * tpt + 1;
-          it.kv_end = max(0, min(L, it.limit0 + it.n_tok - 1));
-          it.slot_off = -1;
-          it.src0 = src_row + t * tpt;
-          it.pad = 0;
-          P.tile_items[e++] = it;
-        }
+    if (P.path_class[p] != kClassDecode) continue;
+    const int rank = P.path_dec_rank[p];
+    const int leaf = P.path_leaf_node[p];
+    const int len = P.node_kv_len[leaf];
+    P.dec_tok[rank] = static_cast<int32_t>(P.q_offsets[p]);
+    P.dec_src[rank] = static_cast<int32_t>(P.q_src_offsets ? P.q_src_offsets[p] : P.q_offsets[p]);
+    P.dec_slot_base[rank] = P.path_slot_base[p];
+    const bool own_leaf = P.node_npaths[leaf] == 1 && len > 0;
+    P.dec_leaf_chunks[rank] = own_leaf ? ceil_div(len, P.leaf_chunk) : 0;
+    for (int g = 0; g < P.Hkv; ++g) P.leaf_arrive[static_cast<int64_t>(rank) * P.Hkv + g] = 0;
+  }
+  // Leaf and chain items, one thread per ITEM (consecutive threads write consecutive descriptors: a thread per path
+  // writing its own run of descriptors makes every store instruction touch 32 different sectors, and that alone cost
+  // tens of microseconds on one SM).  Item e -> path by binary search over the exclusive scans.
+  auto path_of = [&](const int32_t* base, int e) {
+    int lo = 0, hi = live;                    // last p with base[p] <= e (paths without items share their successor's base)
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (base[mid] <= e) lo = mid; else hi = mid;
     }
+    return lo;
+  };
+  const int n_leaf_items = hdr->n_leaf_items;
+  for (int64_t e64 = gtid; e64 < n_leaf_items; e64 += gsize) {
+    const int e = static_cast<int>(e64);
+    const int p = path_of(P.path_leaf_base, e);
+    const int local = e - P.path_leaf_base[p];
+    const int c = local / P.Hkv, g = local - c * P.Hkv;
+    const int leaf = P.path_leaf_node[p];
+    const int len = P.node_kv_len[leaf];
+    LeafItem it;
+    it.page0 = static_cast<int32_t>(P.node_page_offsets[leaf]) + c * (P.leaf_chunk / kPage);
+    it.node = leaf;
+    it.g = g;
+    it.kv_begin = c * P.leaf_chunk;
+    it.kv_end = min(len, (c + 1) * P.leaf_chunk);
+    it.slot = P.path_slot_base[p] + P.node_level_off[leaf] + c;
+    it.q_src = static_cast<int32_t>(P.q_src_offsets ? P.q_src_offsets[p] : P.q_offsets[p]);
+    it.dec = P.path_dec_rank[p];
+    P.leaf_items[e] = it;
+  }
+  const int n_chain_items = hdr->n_tile_items - n_stacked;
+  for (int64_t e64 = gtid; e64 < n_chain_items; e64 += gsize) {
+    const int e = static_cast<int>(e64);
+    const int p = path_of(P.path_chain_base, e);
+    const int local = e - P.path_chain_base[p];
+    const int T = P.path_q_len[p];
+    const int L = P.path_kv_len[p];
+    const int tiles = ceil_div(T, tpt);
+    const int g = local / tiles, t = local - g * tiles;
+    const int32_t src_row = static_cast<int32_t>(P.q_src_offsets ? P.q_src_offsets[p] : P.q_offsets[p]);
+    TileItem it;
+    it.node = P.path_leaf_node[p];
+    it.tok0 = static_cast<int32_t>(P.q_offsets[p]) + t * tpt;
+    it.n_tok = min(tpt, T - t * tpt);
+    it.kind_g = (kItemChain << 16) | g;
+    it.kv_begin = 0;
+    it.limit0 = L - T + t * tpt + 1;
+    it.kv_end = max(0, min(L, it.limit0 + it.n_tok - 1));
+    it.slot_off = -1;
+    it.src0 = src_row + t * tpt;
+    {                                           // page segments of the chain, root first
+      int chain[SS_MAX_DEPTH];
+      int d = 0;
+      for (int a = it.node; a >= 0 && d < SS_MAX_DEPTH; a = P.node_parent[a]) chain[d++] = a;
+      int n_seg = 0, first = 0;
+      it.seg_first[0] = it.seg_first[1] = 0x7fffffff;
+      it.seg_off[0] = it.seg_off[1] = it.seg_off[2] = 0;
+      for (int c = d - 1; c >= 0; --c) {
+        const int n = chain[c];
+        const int np = (P.node_kv_len[n] + kPage - 1) / kPage;
+        if (np == 0) continue;
+        if (n_seg < kItemSegs) {
+          it.seg_off[n_seg] = static_cast<int32_t>(P.node_page_offsets[n]);
+          if (n_seg > 0) it.seg_first[n_seg - 1] = first;
+        }
+        first += np;
+        ++n_seg;
+      }
+      it.n_seg = n_seg <= kItemSegs ? n_seg : -1;
+    }
+    P.tile_items[n_stacked + e] = it;
   }
 
   // stacked items: item e -> node by binary search over the exclusive scan of per-node item counts
@@ -353,12 +388,118 @@ __global__ void __launch_bounds__(kGridThreads) plan_emit_kernel(const Params P)
     it.limit0 = it.kv_end;
     it.slot_off = P.node_level_off[n] + split;
     it.src0 = 0;
-    it.pad = 0;
+    it.n_seg = 1;
+    it.seg_first[0] = it.seg_first[1] = 0x7fffffff;
+    it.seg_off[0] = static_cast<int32_t>(P.node_page_offsets[n]);
+    it.seg_off[1] = it.seg_off[2] = 0;
     P.tile_items[e] = it;
   }
 }
 
+// ---- general path: four launches ------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kGridThreads) plan_nodes_kernel(const Params P) {
+  ss::grid_dependency_enter();
+  plan_nodes_phase(P);
+}
+__global__ void __launch_bounds__(kGridThreads) plan_paths_kernel(const Params P) {
+  ss::grid_dependency_enter();
+  if (P.hdr->status != SS_OK) return;          // no barrier in this kernel: a per-thread return is safe
+  plan_paths_phase(P);
+}
+__global__ void __launch_bounds__(kScanThreads) plan_scan_kernel(const Params P) {
+  ss::grid_dependency_enter();
+  plan_scan_phase(P);
+}
+__global__ void __launch_bounds__(kGridThreads) plan_emit_kernel(const Params P) {
+  ss::grid_dependency_enter();
+  if (P.hdr->status != SS_OK) return;          // no barrier in this kernel
+  plan_emit_phase(P);
+}
+
+// ---- small trees: one block, everything in shared memory -------------------------------------------------------------
+constexpr int kSmallPlan = 2048;               // nodes and paths
+constexpr int kSmallNodeArrays = 11, kSmallPathArrays = 6;
+// bytes of shared memory for N nodes and NP paths: staged inputs + redirected plan arrays
+inline size_t small_plan_smem(int N, int NP) {
+  return static_cast<size_t>(N + 1) * (8 + 4 + 4 + 4 * kSmallNodeArrays) + static_cast<size_t>(NP + 1) * (4 + 4 + 4 * kSmallPathArrays) + 64;
+}
+
+__global__ void __launch_bounds__(kScanThreads) plan_small_kernel(const Params P0) {
+  ss::grid_dependency_enter();
+  extern __shared__ __align__(16) uint8_t plan_smem[];
+  __shared__ PlanHeader s_hdr;       // the header is built here too and written out once, at the end
+  __shared__ int s_live;
+  const int tid = threadIdx.x, nt = blockDim.x;
+  const int N = P0.num_nodes, NP = P0.num_paths;
+  Params P = P0;
+  for (int x = tid; x < static_cast<int>(sizeof(PlanHeader) / 4); x += nt) reinterpret_cast<int32_t*>(&s_hdr)[x] = 0;
+  if (tid == 0) s_live = live_paths(P0);
+  P.hdr = &s_hdr;
+  P.num_paths_dev = &s_live;
+  __syncthreads();
+  SS_STAMP_BEGIN(P.hdr, 0);
+  // carve: 8-byte array first, then 4-byte arrays of N + 1 and of NP + 1 entries
+  int64_t* s_page_off = reinterpret_cast<int64_t*>(plan_smem);
+  int32_t* w = reinterpret_cast<int32_t*>(s_page_off + (N + 1));
+  auto take = [&](int n) { int32_t* p = w; w += n; return p; };
+  int32_t* s_parent = take(N + 1);
+  int32_t* s_len = take(N + 1);
+  int32_t** node_arrays[kSmallNodeArrays] = {&P.node_start, &P.node_depth, &P.node_first, &P.node_last, &P.node_npaths,
+                                             &P.node_ndec, &P.node_own_slots, &P.node_level_off, &P.node_item_base,
+                                             &P.node_splits, &P.node_split_len};
+  for (int i = 0; i < kSmallNodeArrays; ++i) *node_arrays[i] = take(N + 1);
+  int32_t* s_leaf = take(NP + 1);
+  int32_t* s_qlen = take(NP + 1);
+  int32_t** path_arrays[kSmallPathArrays] = {&P.path_class, &P.path_kv_len, &P.path_dec_rank, &P.path_slot_base,
+                                             &P.path_leaf_base, &P.path_chain_base};
+  for (int i = 0; i < kSmallPathArrays; ++i) *path_arrays[i] = take(NP + 1);
+  // stage the tree and the per-path arrays (one round trip; every later chain walk stays on chip)
+  for (int n = tid; n < N; n += nt) { s_parent[n] = P0.node_parent[n]; s_len[n] = P0.node_kv_len[n]; }
+  for (int n = tid; n <= N; n += nt) s_page_off[n] = P0.node_page_offsets[n];
+  const int live = s_live;
+  for (int p = tid; p < live; p += nt) { s_leaf[p] = P0.path_leaf_node[p]; s_qlen[p] = P0.path_q_len[p]; }
+  P.node_parent = s_parent;
+  P.node_kv_len = s_len;
+  P.node_page_offsets = s_page_off;
+  P.path_leaf_node = s_leaf;
+  P.path_q_len = s_qlen;
+  __syncthreads();
+
+  plan_nodes_phase(P);
+  bool failed = block_failed(P.hdr);
+  if (!failed) {
+    plan_paths_phase(P);
+    __syncthreads();
+    plan_scan_phase(P);
+    failed = block_failed(P.hdr);
+  }
+  if (!failed) {
+    plan_emit_phase(P);
+    // the executors read these three from the workspace (exact second pass, generic rows)
+    for (int n = tid; n < N; n += nt) P0.node_start[n] = P.node_start[n];
+    for (int p = tid; p < live; p += nt) { P0.path_class[p] = P.path_class[p]; P0.path_kv_len[p] = P.path_kv_len[p]; }
+  }
+  SS_STAMP_END(P.hdr, 1);
+  __syncthreads();
+  for (int x = tid; x < static_cast<int>(sizeof(PlanHeader) / 4); x += nt)
+    reinterpret_cast<int32_t*>(P0.hdr)[x] = reinterpret_cast<const int32_t*>(&s_hdr)[x];
+}
+
 int32_t launch_plan(const Params& P, cudaStream_t st) {
+  if (P.num_nodes <= kSmallPlan && P.num_paths <= kSmallPlan) {     // (this kernel writes the whole header itself)
+    static bool configured[kDeviceSlots] = {false};
+    const int dev_slot = current_device_slot();
+    if (dev_slot < 0 || !configured[dev_slot]) {
+      if (cudaFuncSetAttribute(plan_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               static_cast<int>(small_plan_smem(kSmallPlan, kSmallPlan))) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return SS_ERR_CUDA;
+      }
+      if (dev_slot >= 0) configured[dev_slot] = true;
+    }
+    SS_LAUNCH(plan_small_kernel, 1, kScanThreads, small_plan_smem(P.num_nodes, P.num_paths), st, P);
+    return SS_OK;
+  }
   if (cudaMemsetAsync(P.hdr, 0, sizeof(PlanHeader), st) != cudaSuccess) {
     (void)cudaGetLastError();
     return SS_ERR_CUDA;

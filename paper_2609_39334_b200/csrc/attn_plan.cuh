@@ -20,15 +20,15 @@ constexpr int kHeadDim = 128;
 constexpr int kPage = 16;
 constexpr int kTileRows = 128;          // stacked rows of one tile item
 constexpr int kKvTile = 64;             // keys per tensor-core step
-constexpr int kLeafChunk = 256;         // keys per leaf item (decode)
+constexpr int kLeafChunk = 256;         // most keys per leaf item (decode); small calls use 128 or 64, see Params::leaf_chunk
 constexpr int kMaxRootSplits = 8;       // KV splits of a root node when there are few tiles
 constexpr int kMinSplitLen = 512;       // a split is at least this many keys
 
 enum PathClass : int32_t { kClassDecode = 0, kClassChain = 1, kClassGeneric = 2 };
 enum ItemKind : int32_t { kItemStacked = 0, kItemChain = 1 };
 
-// One tile of stacked query rows against a KV source.  40 bytes.
-struct TileItem {
+// One tile of stacked query rows against a KV source.  64 bytes.
+struct alignas(8) TileItem {
   int32_t node;       // stacked: the shared node; chain: the path's leaf node
   int32_t tok0;       // stacked: index into dec_tok[]; chain: first query row (global token index)
   int32_t n_tok;      // tokens in the tile (rows = n_tok * G)
@@ -38,19 +38,26 @@ struct TileItem {
   int32_t limit0;     // keys visible to the tile's first token; token i sees limit0 + i * (kind == chain)
   int32_t slot_off;   // stacked: partial slot relative to the token's slot base; chain: -1 (final output)
   int32_t src0;       // chain: row of q holding the tile's first token (stacked: rows come from dec_src[])
-  int32_t pad;
+  // The page segments of the source, so that the kernel need not walk the tree: segment d covers the virtual pages
+  // [seg_first[d], seg_first[d + 1]) of the key sequence (seg_first[0] = 0) and starts at node_pages[seg_off[d]].
+  // A stacked item has one segment (its node); a chain item one per non-empty node root -> leaf.  n_seg = -1: more
+  // than kItemSegs segments, the kernel walks the chain itself.
+  int32_t n_seg;
+  int32_t seg_first[2];   // of segments 1 and 2
+  int32_t seg_off[3];
 };
+constexpr int kItemSegs = 3;
 
 // One chunk of a decode path's private leaf.  32 bytes.
-struct LeafItem {
-  int32_t q_row;      // global query token index
+struct alignas(16) LeafItem {
+  int32_t page0;      // index into node_pages of the chunk's first page
   int32_t node;       // leaf node
   int32_t g;          // kv head
   int32_t kv_begin;   // token range inside the leaf
   int32_t kv_end;
   int32_t slot;       // absolute partial slot
   int32_t q_src;      // row of q holding the token's query
-  int32_t pad1;
+  int32_t dec;        // decode rank of the token (index into dec_tok / dec_slot_base / dec_leaf_chunks)
 };
 
 struct PlanHeader {       // first bytes of the workspace; status MUST be the first word
@@ -65,7 +72,25 @@ struct PlanHeader {       // first bytes of the workspace; status MUST be the fi
   int32_t leaf_counter;
   int32_t n_stacked_items; // tile items [0, n_stacked_items) are stacked items, the rest chain items
   int32_t pad[6];
+#ifdef SS_STAMPS
+  unsigned long long stamp[8];   // instrumented build: %globaltimer at kernel starts / ends (see SS_STAMP)
+#endif
 };
+
+// Instrumented build (-DSS_STAMPS): the first thread of a kernel records when it started (after its predecessor
+// completed), every block when it ended; slots 0/1 planner, 2/3 tile kernel, 4/5 leaf kernel, 6/7 merge.
+#ifdef SS_STAMPS
+__device__ __forceinline__ unsigned long long ss_globaltimer() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+#define SS_STAMP_BEGIN(hdr, i) do { if (blockIdx.x == 0 && threadIdx.x == 0) (hdr)->stamp[i] = ss_globaltimer(); } while (0)
+#define SS_STAMP_END(hdr, i) do { if (threadIdx.x == 0) atomicMax(&(hdr)->stamp[i], ss_globaltimer()); } while (0)
+#else
+#define SS_STAMP_BEGIN(hdr, i) do { } while (0)
+#define SS_STAMP_END(hdr, i) do { } while (0)
+#endif
 
 struct Caps {             // host-computed capacities of the plan arrays
   int32_t dec, tile_items, leaf_items;
@@ -94,6 +119,8 @@ struct Params {
   __nv_bfloat16* out;
   float* lse;
   int32_t target_tiles;      // the planner splits root nodes until about this many tile items exist
+  int32_t leaf_chunk;        // keys per leaf item: 256, or less when the call is too small to keep every warp of the
+                             // leaf kernel supplied with several items (chosen on the host from the page count)
   Caps caps;
   // ---- workspace regions ----
   PlanHeader* hdr;
@@ -101,6 +128,8 @@ struct Params {
       *node_level_off, *node_item_base, *node_splits, *node_split_len;
   int32_t *path_class, *path_kv_len, *path_dec_rank, *path_slot_base, *path_leaf_base, *path_chain_base;
   int32_t *dec_tok, *dec_src, *dec_slot_base;   // per decode token: output row, query row, first partial slot
+  int32_t *dec_leaf_chunks;  // per decode token: leaf items per kv head (0: empty or shared leaf)
+  int32_t *leaf_arrive;      // [decode token][kv head]: leaf items that have written their partial (zeroed by the planner)
   TileItem* tile_items;
   LeafItem* leaf_items;
   float* part_o;             // [slots][Hq][128]

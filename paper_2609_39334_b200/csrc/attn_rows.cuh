@@ -105,5 +105,105 @@ __device__ __forceinline__ void tile_item_rows_exact(const Params& P, const Tile
   }
 }
 
+// Log-sum-exp merge of the per-level partial results of decode token `d`, q head `h` (one whole warp):
+// out = sum_s exp(lse_s - LSE) o_s,  LSE = log sum_s exp(lse_s); a token without partials (no keys) gives 0 / -inf.
+// The partials are read from L2 (ld.global.cg): inside the leaf kernel they may have been written by other SMs
+// moments ago.
+__device__ __forceinline__ void merge_row(const Params& P, int d, int h, int lane) {
+  const int s0 = P.dec_slot_base[d], s1 = P.dec_slot_base[d + 1];
+  float m = -INFINITY;
+  for (int s = s0 + lane; s < s1; s += 32) m = fmaxf(m, __ldcg(P.part_lse + static_cast<int64_t>(s) * P.Hq + h));
+  m = warp_max(m);
+  RowState r;
+  r.acc[0] = r.acc[1] = r.acc[2] = r.acc[3] = 0.f;
+  r.l = 0.f;
+  r.m = m;
+  if (m > -INFINITY) {
+    for (int s = s0; s < s1; ++s) {
+      const float ls = __ldcg(P.part_lse + static_cast<int64_t>(s) * P.Hq + h);
+      if (ls == -INFINITY) continue;
+      const float wgt = __expf(ls - m);
+      const float4 o = __ldcg(reinterpret_cast<const float4*>(P.part_o + (static_cast<int64_t>(s) * P.Hq + h) * kHeadDim + 4 * lane));
+      r.l += wgt;
+      r.acc[0] += wgt * o.x; r.acc[1] += wgt * o.y; r.acc[2] += wgt * o.z; r.acc[3] += wgt * o.w;
+    }
+  }
+  row_store_final(r, P, P.dec_tok[d], h, lane);
+}
+
+// The same merge for the (up to 8) q heads [h0, h0 + n_rows) of decode token `d` at once (one whole warp).  The rows
+// are independent, so their loads are issued together: merging them one after another costs two memory round trips
+// per row, which is what a leaf item's last warp would otherwise wait for.
+__device__ __forceinline__ void merge_rows8(const Params& P, int d, int h0, int n_rows, int lane) {
+  const int s0 = P.dec_slot_base[d], s1 = P.dec_slot_base[d + 1];
+  float m[8];
+#pragma unroll
+  for (int r = 0; r < 8; ++r) {
+    m[r] = -INFINITY;
+    if (r < n_rows)
+      for (int s = s0 + lane; s < s1; s += 32) m[r] = fmaxf(m[r], __ldcg(P.part_lse + static_cast<int64_t>(s) * P.Hq + h0 + r));
+  }
+#pragma unroll
+  for (int r = 0; r < 8; ++r) m[r] = warp_max(m[r]);
+  float acc[8][4], l[8];
+#pragma unroll
+  for (int r = 0; r < 8; ++r) { acc[r][0] = acc[r][1] = acc[r][2] = acc[r][3] = 0.f; l[r] = 0.f; }
+  for (int s = s0; s < s1; ++s) {
+    float ls[8];
+    float4 o[8];
+#pragma unroll
+    for (int r = 0; r < 8; ++r) {
+      ls[r] = -INFINITY;
+      o[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (r < n_rows) {
+        ls[r] = __ldcg(P.part_lse + static_cast<int64_t>(s) * P.Hq + h0 + r);
+        o[r] = __ldcg(reinterpret_cast<const float4*>(P.part_o + (static_cast<int64_t>(s) * P.Hq + h0 + r) * kHeadDim + 4 * lane));
+      }
+    }
+#pragma unroll
+    for (int r = 0; r < 8; ++r) {
+      const float wgt = ls[r] == -INFINITY ? 0.f : __expf(ls[r] - m[r]);   // (m = -inf only if every ls is)
+      l[r] += wgt;
+      acc[r][0] += wgt * o[r].x; acc[r][1] += wgt * o[r].y; acc[r][2] += wgt * o[r].z; acc[r][3] += wgt * o[r].w;
+    }
+  }
+  const int64_t q_row = P.dec_tok[d];
+#pragma unroll
+  for (int r = 0; r < 8; ++r) {
+    if (r >= n_rows) continue;
+    RowState rs;
+    rs.acc[0] = acc[r][0]; rs.acc[1] = acc[r][1]; rs.acc[2] = acc[r][2]; rs.acc[3] = acc[r][3];
+    rs.l = l[r];
+    rs.m = m[r];
+    row_store_final(rs, P, q_row, h0 + r, lane);
+  }
+}
+
+// Rows of GENERIC paths: warp `w` of `warps` takes rows w, w + warps, ... of all (query token, q head) rows.
+__device__ inline void generic_rows(const Params& P, int64_t w, int64_t warps, int lane) {
+  const int live = P.hdr->live_paths;
+  if (live <= 0) return;
+  const int64_t total_rows = P.q_offsets[live] * P.Hq;
+  for (; w < total_rows; w += warps) {
+    const int64_t q_row = w / P.Hq;
+    const int h = static_cast<int>(w % P.Hq);
+    int lo = 0, hi = live;                    // path with q_offsets[p] <= q_row < q_offsets[p+1]
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (P.q_offsets[mid] <= q_row) lo = mid; else hi = mid;
+    }
+    const int p = lo;
+    if (P.path_class[p] != kClassGeneric) continue;
+    const int T = P.path_q_len[p];
+    const int t = static_cast<int>(q_row - P.q_offsets[p]);
+    const int visible = P.path_kv_len[p] - T + t + 1;
+    RowState r;
+    const int64_t q_src = P.q_src_offsets ? P.q_src_offsets[p] + t : q_row;
+    row_init(r, P.q + (q_src * P.Hq + h) * kHeadDim, lane);
+    if (visible > 0) row_visit_chain(r, P, P.path_leaf_node[p], h / P.G, 0, visible, lane);
+    row_store_final(r, P, q_row, h, lane);
+  }
+}
+
 }  // namespace attn
 }  // namespace ss

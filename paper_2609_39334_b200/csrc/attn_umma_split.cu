@@ -144,6 +144,7 @@ tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const _
   ss::grid_dependency_enter();
   extern __shared__ __align__(1024) uint8_t smem[];
   __shared__ Ctrl C;
+  SS_STAMP_BEGIN(P.hdr, 2);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   volatile int* abort_flag = &C.abort_flag;
 
@@ -683,6 +684,7 @@ tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const _
     __syncthreads();
   }
   if (warp == kSoftmaxWarps) tmem_dealloc(tmem, kTmemCols);
+  SS_STAMP_END(P.hdr, 3);
 }
 
 }  // namespace split

@@ -20,7 +20,25 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 
 OUT_MAX, OUT_MEAN, LSE_MAX = 2e-2, 2e-3, 1e-3          # official
-TIGHT_OUT_MAX, TIGHT_OUT_MEAN, TIGHT_LSE = 6e-3, 4e-4, 2e-4   # internal, random N(0,1) data
+# Internal gates, set from the errors observed on a B200 (SS_PARITY_LOG collects them):
+#   * paths of >= 256 keys (every benchmark configuration): observed out max <= 9.8e-4, mean <= 1.1e-4 -> 4e-3 / 3e-4;
+#   * any length, element by element: |err| <= 2^-8 |exact| + 2.5e-3.  The bf16 rounding of the output is at most 2^-9
+#     relative; rounding P to bf16 before P V perturbs every term p_j v_j by up to 2^-9 relative, which does not shrink
+#     with |exact| when terms cancel: with a few dominant keys and |v| up to ~4 that is up to a few 1e-3 (observed:
+#     1.4e-3 beyond the relative part on 100-key verification rows, 5.4e-3 in all on 5-key paths with outputs near 3);
+#   * LSE: fp32 sums of ex2.approx values, observed <= 2.6e-6 -> 2e-5 (a causal mask that is off by one key moves the LSE
+#     of a 4672-key row by 2e-4).
+TIGHT_OUT_MAX, TIGHT_OUT_MEAN, TIGHT_LSE = 4e-3, 3e-4, 2e-5
+TIGHT_REL, TIGHT_ABS = 2.0 ** -8, 2.5e-3
+LONG_PATH = 256
+
+
+def tight_gates(out, o_ref, lerr, min_len):
+    err = np.abs(out - o_ref)
+    assert (err <= TIGHT_REL * np.abs(o_ref) + TIGHT_ABS).all(), float((err - TIGHT_REL * np.abs(o_ref)).max())
+    assert lerr <= TIGHT_LSE, lerr
+    if min_len >= LONG_PATH:
+        assert err.max() <= TIGHT_OUT_MAX and err.mean() <= TIGHT_OUT_MEAN, (err.max(), err.mean())
 
 
 def log_observed(name, out_max, out_mean, lse_max):
@@ -82,12 +100,11 @@ def check_attention(r, w, ref, max_paths=48, tight=True, host_w=None):
     log_observed(f"{w.name} tight={tight}", err.max(), err.mean(), lerr)
     assert err.max() <= OUT_MAX and err.mean() <= OUT_MEAN and lerr <= LSE_MAX, (err.max(), err.mean(), lerr)
     if tight:
-        assert err.max() <= TIGHT_OUT_MAX and err.mean() <= TIGHT_OUT_MEAN and lerr <= TIGHT_LSE, \
-            (err.max(), err.mean(), lerr)
+        tight_gates(out, o_ref, lerr, min(src.path_kv_len(int(u)) for u in uniq))
     return err.max(), err.mean(), lerr
 
 
-MODES = [("fast", 0), ("two_cta", B.SS_FLAG_TILES_2CTA), ("no_tcgen05", B.SS_FLAG_NO_TCGEN05),
+MODES = [("fast", 0), ("flow", B.SS_FLAG_TILES_FLOW), ("two_cta", B.SS_FLAG_TILES_2CTA), ("no_tcgen05", B.SS_FLAG_NO_TCGEN05),
          ("generic", B.SS_FLAG_FORCE_GENERIC)]
 
 
@@ -376,7 +393,7 @@ def test_attention_page_permutation_and_explicit_scale():
     w = synth.build_tree_workload("perm", 5, 12, 2, [128], [6], 2, (1, 120), lambda i, n, rng: 1 + (i % 2) * 30)
     r1, ref = attention_only(w, sm_scale=0.05)
     o_ref, l_ref = oracle.tree_attention_workload(w, paths=ref["unique_paths"], sm_scale=0.05)
-    assert np.abs(r1["out"] - o_ref).max() <= TIGHT_OUT_MAX and np.abs(r1["lse"] - l_ref).max() <= TIGHT_LSE
+    tight_gates(r1["out"], o_ref, np.abs(r1["lse"] - l_ref).max(), 0)
     rng = np.random.default_rng(0)
     perm = rng.permutation(w.num_pages)
     new_pool = torch.empty_like(w.kv_pool)
@@ -384,8 +401,8 @@ def test_attention_page_permutation_and_explicit_scale():
     w.kv_pool = new_pool
     w.node_pages = perm[w.node_pages].astype(np.int32)
     r2, _ = attention_only(w, sm_scale=0.05)
-    assert np.abs(r2["out"] - r1["out"]).max() <= 2 * TIGHT_OUT_MAX
-    assert np.abs(r2["lse"] - r1["lse"]).max() <= 2 * TIGHT_LSE
+    # only the physical page ids differ: every item sees the same numbers in the same order
+    assert np.array_equal(r2["out"], r1["out"]) and np.array_equal(r2["lse"], r1["lse"])
 
 
 def test_attention_empty_and_degenerate():
@@ -455,7 +472,7 @@ def test_config5_full_size_sampled_outputs():
     lerr = np.abs(lse - l_ref).max()
     log_observed("config5_full", err.max(), err.mean(), lerr)
     assert err.max() <= OUT_MAX and err.mean() <= OUT_MEAN and lerr <= LSE_MAX, (err.max(), err.mean(), lerr)
-    assert err.max() <= TIGHT_OUT_MAX and err.mean() <= TIGHT_OUT_MEAN and lerr <= TIGHT_LSE, (err.max(), err.mean(), lerr)
+    tight_gates(out, o_ref, lerr, LONG_PATH)
 
 
 def test_attention_without_query_indirection_matches():
