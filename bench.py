@@ -178,6 +178,25 @@ def time_oracle(w_host, steps, warmup):
 # ------------------------------------------------------------------------------------------------------------
 # the smaller benchmark configurations and the "next" rows, reported inside the default run's JSON line
 # ------------------------------------------------------------------------------------------------------------
+class L2Flush:
+    """Evicts L2 between timed iterations: a buffer of twice the L2 size is written, then a second one is read, so that
+    the cache ends up full of CLEAN lines of data the step never touches.  (After a write alone, half of the buffer
+    sits in L2 as dirty lines, and the step under test pays for their write-back: 126 MB of extra DRAM traffic inside
+    the timed region, half as much again as a small configuration reads.)"""
+    NOTE = "L2 flushed between iterations (252 MB written, then 252 MB read: no dirty lines left)"
+
+    def __init__(self, dev):
+        import torch
+        self.w = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=dev)
+        self.r = torch.zeros(2 * L2_BYTES // 4, dtype=torch.int32, device=dev)
+        self.sink = torch.zeros((), dtype=torch.int64, device=dev)
+
+    def fill_(self, i):
+        import torch
+        self.w.fill_(i & 0xff)
+        torch.sum(self.r, dim=(0,), out=self.sink)
+
+
 def timed_ms(fn, steps, flush, dev):
     """CUDA-event time of `fn` per call, `steps` calls, L2 evicted before each (outside the events)."""
     import torch
@@ -237,7 +256,7 @@ def small_workload(name, dev, flush, peaks, steps=20, warmup=5):
            "phase_ms": phases,
            "phase_note": "phase times carry the profiler's events (a few microseconds each); the attention and step "
                          "times above are measured without them",
-           "l2": "L2 flushed between iterations", "steps": steps, "warmup": warmup, "clocks": clk}
+           "l2": L2Flush.NOTE, "steps": steps, "warmup": warmup, "clocks": clk}
     if phases.get("tiles"):
         ach = work["tile_flops"] / (phases["tiles"] * 1e-3) / 1e12
         out["tiles"] = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_burst"], "unit": "TFLOP/s",
@@ -372,11 +391,11 @@ def lv_sweep(args):
     torch.cuda.set_device(dev)
     if int(os.environ.get("RANK", "0")) != 0:
         return
-    flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=dev)
+    flush = L2Flush(dev)
     curve, knee = lv_curve(dev, flush, args.steps, args.warmup)
     print(json.dumps({"metric": "verification_attention_step_tokens_per_s", "unit": "tokens/s", "n_gpus": 1,
                       "steps": args.steps, "warmup": max(args.warmup, 3), "dtype": "bf16", "data": "synthetic",
-                      "config": {"workload": "lv-sweep", "heads": "28q/4kv", "prefix": 1024, "l2": "L2 flushed between iterations"},
+                      "config": {"workload": "lv-sweep", "heads": "28q/4kv", "prefix": 1024, "l2": L2Flush.NOTE},
                       "curve": curve, "knee_tokens_at_90pct": knee,
                       "paper_context": "the paper's reward-model forward saturates near 2048 batched tokens on an A100 "
                                        "(Section Lazy Verification); this curve is the attention call alone on a B200"}))
@@ -393,7 +412,6 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--tiles-2cta", action="store_true",
                     help="run the tile items on the two-CTAs-per-SM kernel (64-key tiles) instead of the default one")
-    ap.add_argument("--tiles-flow", action="store_true", help="run the tile items on the free-running kernel")
     ap.add_argument("--graph", action="store_true",
                     help="also time the step as a CUDA graph replay (reported as ms_per_step_cuda_graph)")
     ap.add_argument("--no-e2e", action="store_true")
@@ -462,11 +480,11 @@ def main():
     # every rank its own problems: same shapes, different seed
     from paper_2609_39334_b200 import replicas
     w = replicas.replica_workload(synth.make_config, cfg_idx, rank, device=dev, scale=args.scale, poison=True)
-    pipe = DevicePipeline(w, dev, attn_flags=B.SS_FLAG_TILES_2CTA if args.tiles_2cta else (B.SS_FLAG_TILES_FLOW if args.tiles_flow else 0))
+    pipe = DevicePipeline(w, dev, attn_flags=B.SS_FLAG_TILES_2CTA if args.tiles_2cta else 0)
     kv_bytes = pipe.kv_pool.numel() * 2
     flush = None
     if kv_bytes < 4 * L2_BYTES:
-        flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=dev)
+        flush = L2Flush(dev)
 
     def sync_all():
         torch.cuda.synchronize(dev)
@@ -594,7 +612,7 @@ def main():
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": args.workload, "paths": w.num_paths, "unique_paths": U, "query_tokens": tokens,
                    "heads": f"{w.num_q_heads}q/{w.num_kv_heads}kv", "kv_pool_gb": kv_bytes / 1e9,
-                   "l2": "inputs larger than L2" if flush is None else "L2 flushed between iterations",
+                   "l2": "inputs larger than L2" if flush is None else L2Flush.NOTE,
                    "parallelism": f"replicas x{world}" if world > 1 else "single GPU"},
         "gpu_launches": int(launches),
         "attention_ms_per_step": attn_ms,
@@ -613,6 +631,7 @@ def main():
     if not args.no_e2e:
         from paper_2609_39334_b200.pipeline import HostStepPipeline
         host = HostStepPipeline(pipe, depth=args.e2e_depth)
+        slim = host.measure_traffic()                     # (bytes per step as the call really moves them)
         for i in range(args.e2e_depth):
             host.submit(i)
         host.synchronize()
@@ -636,9 +655,12 @@ def main():
                       "h2d_bytes_per_step": int(host.h2d_bytes), "d2h_bytes_per_step": int(host.d2h_bytes),
                       "ms_per_step": e2e_ms, "steps": n_e2e, "sets_in_flight": args.e2e_depth,
                       "api": "ss_candidate_step_host",
-                      "note": "KV pool stays resident (it is the cache); every step copies candidates, queries and "
-                              "scores from pinned host memory and all results back; steps alternate between "
-                              "independent (host buffers, device arena, stream) sets so copies overlap kernels"}
+                      "unique_rows_only": bool(slim),
+                      "note": "KV pool stays resident (it is the cache); every step copies candidates and scores from "
+                              "pinned host memory, fetches the query rows of the unique paths from it after the "
+                              "deduplication and writes the live rows of out / lse and all other results back; steps "
+                              "alternate between independent (host buffers, device arena, stream) sets so copies "
+                              "overlap kernels"}
         del host
 
     # ---- CPU oracle beside it (rank 0, N = 1 only) ----------------------------------------------------------------
@@ -660,7 +682,7 @@ def main():
         w.kv_pool = None
         w.q = None
         torch.cuda.empty_cache()
-        small_flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=dev)
+        small_flush = L2Flush(dev)
         out["workloads"] = {name: small_workload(name, dev, small_flush, peaks) for name in ("c2", "c3", "c4")}
         out["next_rows"] = next_rows(dev, small_flush, peaks)
         curve, knee = lv_curve(dev, small_flush, 20, 3)

@@ -54,8 +54,6 @@ extern "C" {
 #define SS_FLAG_TILES_2CTA 0x10u    /* attention: run the tcgen05 tile items on the kernel that keeps two CTAs
                                        per SM and works on 64-key tiles (default: the one-CTA-per-SM kernel with
                                        128-key tiles); same results within the accuracy contract             */
-#define SS_FLAG_TILES_FLOW 0x20u    /* attention: run the tcgen05 tile items on the free-running kernel (roles do
-                                       not meet at item ends, two accumulators); same results                 */
 
 #define SS_MAX_DEPTH 16             /* maximum number of nodes on a root-to-leaf chain                       */
 
@@ -197,7 +195,9 @@ typedef struct ss_attn_desc {
   int32_t num_q_heads, num_kv_heads; /* Hq % Hkv == 0 */
   int32_t head_dim, page_size;       /* 128, 16 */
   float sm_scale;                    /* 0 => 1/sqrt(head_dim) */
-  int32_t reserved0;
+  int32_t max_sms;                   /* 0: use every SM; otherwise the attention kernels occupy at most this many
+                                        (their blocks need an SM to themselves: a caller that runs long-lived small
+                                        kernels beside the call - copy kernels - leaves those SMs out) */
   const void* k_pool;                /* bf16 */
   const void* v_pool;                /* bf16 */
   int64_t num_pages;                 /* pages addressable through k_pool / v_pool */
@@ -360,6 +360,11 @@ int32_t ss_build_prefix_tree(const int32_t* tok_ids, const int64_t* tok_offsets,
  *   asynchronous copies host -> device of every per-step input  ->  ss_dedup_paths  ->  ss_gather_unique_paths  ->
  *   ss_tree_attention (queries read in place through the gathered offsets)  ->  ss_topk_prune  ->
  *   asynchronous copies device -> host of every result.
+ * If q, out and lse are page-locked AND mapped into the device's address space (memory from cudaHostAlloc or
+ * cudaHostRegister), the rows of duplicate candidates never cross the bus: the queries are fetched after the
+ * deduplication, for the unique paths only, by a small kernel that reads the host buffer directly, and only the
+ * live rows of out / lse (the first u_q_offsets[num_unique]) are written back, again by a kernel; the rest of
+ * out / lse is left untouched.  Buffers that are not mapped are copied whole with cudaMemcpyAsync.
  * Everything is enqueued on `stream`; the call does not synchronise, and it allocates nothing: staging buffers,
  * results and the workspaces of the three calls are carved out of `device_arena` (caller-owned, 256-byte aligned,
  * >= ss_candidate_step_host_arena_bytes).  The KV pool and the tree stay resident on the device: they are the

@@ -29,7 +29,6 @@ SS_FLAG_FORCE_GENERIC = 0x2
 SS_FLAG_NO_TCGEN05 = 0x4
 SS_FLAG_WEAK_HASH = 0x8
 SS_FLAG_TILES_2CTA = 0x10
-SS_FLAG_TILES_FLOW = 0x20
 SS_MAX_DEPTH = 16
 SS_DEDUP_STATIC_MAX_PATHS = 65536
 
@@ -55,7 +54,7 @@ class ss_attn_desc_t(ctypes.Structure):
         ("struct_size", ctypes.c_uint32), ("flags", ctypes.c_uint32),
         ("num_q_heads", ctypes.c_int32), ("num_kv_heads", ctypes.c_int32),
         ("head_dim", ctypes.c_int32), ("page_size", ctypes.c_int32),
-        ("sm_scale", ctypes.c_float), ("reserved0", ctypes.c_int32),
+        ("sm_scale", ctypes.c_float), ("max_sms", ctypes.c_int32),
         ("k_pool", ctypes.c_void_p), ("v_pool", ctypes.c_void_p),
         ("num_pages", ctypes.c_int64),
         ("kv_page_stride", ctypes.c_int64), ("kv_head_stride", ctypes.c_int64), ("kv_token_stride", ctypes.c_int64),

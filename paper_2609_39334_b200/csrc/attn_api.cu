@@ -16,7 +16,6 @@ int32_t launch_merge(const Params& P, cudaStream_t st, int sm_count);
 int32_t launch_leaf_items(const Params& P, cudaStream_t st, int sm_count);
 int32_t launch_tile_items_umma(const Params& P, cudaStream_t st, int sm_count);
 int32_t launch_tile_items_umma_split(const Params& P, cudaStream_t st, int sm_count);
-int32_t launch_tile_items_umma_flow(const Params& P, cudaStream_t st, int sm_count);
 bool leaf_stream_supported(const Params& P);
 int32_t launch_leaf_stream(const Params& P, cudaStream_t st, int sm_count);
 
@@ -61,9 +60,9 @@ static int sm_count_of_current_device() {
 
 static int32_t check_desc(const ss_attn_desc_t* d) {
   if (!d || d->struct_size != sizeof(ss_attn_desc_t)) return SS_ERR_INVALID_ARG;
-  if (d->flags & ~(SS_FLAG_VALIDATE | SS_FLAG_FORCE_GENERIC | SS_FLAG_NO_TCGEN05 | SS_FLAG_TILES_2CTA | SS_FLAG_TILES_FLOW)) return SS_ERR_INVALID_ARG;
+  if (d->flags & ~(SS_FLAG_VALIDATE | SS_FLAG_FORCE_GENERIC | SS_FLAG_NO_TCGEN05 | SS_FLAG_TILES_2CTA)) return SS_ERR_INVALID_ARG;
   if (d->num_q_heads < 1 || d->num_kv_heads < 1 || d->num_nodes < 0 || d->num_paths < 0 || d->total_q < 0 ||
-      d->total_node_pages < 0 || d->num_pages < 0 || d->max_depth < 0 || d->max_decode_paths < 0)
+      d->total_node_pages < 0 || d->num_pages < 0 || d->max_depth < 0 || d->max_decode_paths < 0 || d->max_sms < 0)
     return SS_ERR_INVALID_ARG;
   if (d->head_dim != kHeadDim || d->page_size != kPage) return SS_ERR_UNSUPPORTED;
   if (d->num_q_heads % d->num_kv_heads) return SS_ERR_UNSUPPORTED;
@@ -89,12 +88,9 @@ static Layout carve(const ss_attn_desc_t* d, char* base, Params* P) {
   const int64_t cap_dec = d->max_decode_paths > 0 ? (d->max_decode_paths < d->num_paths ? d->max_decode_paths : d->num_paths)
                                                   : d->num_paths;
   const int target = 2 * sm_count_of_current_device();   // (the size query and the call must see the same device)
-  // Keys per leaf item.  The leaf kernel runs ~12 warps per SM, each a pipeline of its own; with fewer than about eight
-  // items per warp the longest warp sets the kernel's time, so small calls cut the leaves finer (more partials to
-  // merge, which stay in L2).  Decided from host-side numbers only, so that the capacities below match the plan.
-  const int64_t page_items = d->total_node_pages * Hkv;
-  const int64_t warp_slots = 12LL * sm_count_of_current_device();
-  (void)page_items; (void)warp_slots;
+  // Keys per leaf item.  (Finer items - 128 or 64 keys - were measured on the small configurations, where a warp of
+  // the leaf kernel gets fewer than two items: the extra partials, counters and merges cost more than the better
+  // balance gains, 0.50 -> 0.41 of the HBM rate at 64 keys; whole-leaf items of up to 512 keys: no gain either.)
   const int leaf_chunk = kLeafChunk;
   Caps caps;
   caps.dec = static_cast<int32_t>(cap_dec);
@@ -213,7 +209,8 @@ extern "C" int32_t ss_tree_attention(const ss_attn_desc_t* d, void* workspace, s
   P.lse = d->lse;
 
   cudaStream_t st = as_stream(stream);
-  const int sms = sm_count_of_current_device();
+  int sms = sm_count_of_current_device();
+  if (d->max_sms > 0 && d->max_sms < sms) sms = d->max_sms;
   const bool timed = prof_begin_call();
   const int call = g_prof.used;
   // phase boundaries: event e is recorded before phase e, event SS_NUM_PHASES after the last one
@@ -228,9 +225,7 @@ extern "C" int32_t ss_tree_attention(const ss_attn_desc_t* d, void* workspace, s
   if (rc == SS_OK && any && !generic_only) {
     const bool two_cta = (d->flags & SS_FLAG_TILES_2CTA) != 0;
     rc = simple ? launch_tile_items_simple(P, st, sms)
-                : (two_cta ? launch_tile_items_umma(P, st, sms)
-                           : ((d->flags & SS_FLAG_TILES_FLOW) ? launch_tile_items_umma_flow(P, st, sms)
-                                                              : launch_tile_items_umma_split(P, st, sms)));
+                : (two_cta ? launch_tile_items_umma(P, st, sms) : launch_tile_items_umma_split(P, st, sms));
     ran(SS_PHASE_TILES);
   }
   // Decode leaves.  The streaming kernel also merges the per-level partials and computes the rows of GENERIC paths;

@@ -56,7 +56,11 @@ __global__ void __launch_bounds__(kLeafWarps * 32) leaf_items_kernel(const Param
     const int n_keys = it.kv_end - it.kv_begin;
     const int n_pages = (n_keys + kPage - 1) / kPage;                      // <= 16
     const int64_t pg0 = P.node_page_offsets[it.node] + it.kv_begin / kPage;
-    const int my_page = lane < n_pages ? P.node_pages[pg0 + lane] : 0;
+    int my_page = lane < n_pages ? P.node_pages[pg0 + lane] : 0;
+    SS_CHECK_OR(my_page >= 0 && my_page < P.num_pages, &P.hdr->status, my_page = 0);
+    bool slot_ok = true;
+    (void)slot_ok;
+    SS_CHECK_OR(it.slot >= 0 && it.slot < P.caps.slots, &P.hdr->status, slot_ok = false);
 
     // ---- query fragments (dim-permuted, see above) --------------------------------------------------------
     uint4 qa[4], qb[4];
@@ -187,6 +191,9 @@ __global__ void __launch_bounds__(kLeafWarps * 32) leaf_items_kernel(const Param
     for (int rg = 0; rg < (TWO ? 2 : 1); ++rg) {
       const int row = gid + 8 * rg;
       if (row >= G) continue;
+#ifdef SS_CHECKED
+      if (!slot_ok) continue;
+#endif
       const float l = rg ? l1 : l0, m = rg ? m1 : m0;
       const float inv = l > 0.f ? 1.f / l : 0.f;
       const int h = it.g * G + row;

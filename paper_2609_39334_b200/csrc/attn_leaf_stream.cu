@@ -134,6 +134,10 @@ leaf_stream_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     if (!it.valid) return;
     it.g = f_it.g; it.n_keys = f_it.kv_end - f_it.kv_begin; it.slot = f_it.slot; it.dec = f_it.dec;
     it.n_pages = (it.n_keys + kPage - 1) / kPage;               // <= 16
+    SS_CHECK_OR(it.n_keys >= 0 && it.n_pages <= 32 && f_it.page0 >= 0 && f_it.page0 + it.n_pages <= P.total_node_pages &&
+                    it.dec >= 0 && it.dec < P.caps.dec && it.g >= 0 && it.g < P.Hkv && f_it.q_src >= 0 &&
+                    f_it.q_src < (P.q_src_offsets ? P.q_src_rows : P.total_q),
+                &P.hdr->status, { it.valid = 0; return; });
     it.my_page = lane < it.n_pages ? P.node_pages[static_cast<int64_t>(f_it.page0) + lane] : 0;
     it.chunks = P.dec_leaf_chunks[f_it.dec];
     // B fragments of Q^T: thread (gid, tig) holds Q[row 8 nt + gid][dims 16 ks + 2 tig, + 1] and the same 8 dims on
@@ -161,7 +165,8 @@ leaf_stream_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     if (n_issued - n_cons >= static_cast<uint32_t>(kStages)) return;
     if (!prod_in_next && prod_pg >= cur.n_pages) { prod_in_next = true; prod_pg = 0; }
     if (prod_in_next && (!nxt.valid || prod_pg >= nxt.n_pages)) return;
-    const int page = __shfl_sync(0xffffffffu, prod_in_next ? nxt.my_page : cur.my_page, prod_pg);
+    int page = __shfl_sync(0xffffffffu, prod_in_next ? nxt.my_page : cur.my_page, prod_pg);
+    SS_CHECK_OR(page >= 0 && page < P.num_pages, &P.hdr->status, page = 0);
     const int g = prod_in_next ? nxt.g : cur.g;
     const int stage = n_issued % kStages;
     if (lane == 0) {
@@ -317,8 +322,11 @@ leaf_stream_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       // The leaf is this one item: nothing else will arrive for the (token, kv head), and the shared-node partials are
       // complete (the tile kernel ran before).  Fold them into the accumulator registers and write the final rows -
       // no partial of its own, no fence, no counter, no second pass over what was just written.
-      const int s0 = P.dec_slot_base[cur.dec], s1 = P.dec_slot_base[cur.dec + 1];
+      int s0 = P.dec_slot_base[cur.dec], s1 = P.dec_slot_base[cur.dec + 1];
       const int64_t q_row = P.dec_tok[cur.dec];
+      bool row_ok = true;
+      SS_CHECK_OR(s0 >= 0 && s0 <= s1 && s1 <= P.caps.slots, &P.hdr->status, s1 = s0);
+      SS_CHECK_OR(q_row >= 0 && q_row < P.total_q, &P.hdr->status, row_ok = false);
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
@@ -356,17 +364,19 @@ leaf_stream_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             const float lo = o[mt][nt][x] * inv, hi = o[mt][nt][2 + x] * inv;
             const float got = __shfl_xor_sync(0xffffffffu, (gid & 1) ? lo : hi, 4);
             const uint32_t pk = (gid & 1) ? pack_bf16(got, hi) : pack_bf16(lo, got);
-            if (q_live) *reinterpret_cast<uint32_t*>(dst + 16 * mt) = pk;
+            if (q_live && row_ok) *reinterpret_cast<uint32_t*>(dst + 16 * mt) = pk;
           }
-          if (q_live && gid == 0 && P.lse) P.lse[q_row * P.Hq + h] = den > 0.f ? big + __logf(den) : -INFINITY;
+          if (q_live && row_ok && gid == 0 && P.lse) P.lse[q_row * P.Hq + h] = den > 0.f ? big + __logf(den) : -INFINITY;
         }
     } else {
+      bool slot_ok = true;
+      SS_CHECK_OR(cur.slot >= 0 && cur.slot < P.caps.slots, &P.hdr->status, slot_ok = false);
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
         for (int x = 0; x < 2; ++x) {
           const int q = 8 * nt + 2 * tig + x;
-          if (q >= G) continue;
+          if (q >= G || !slot_ok) continue;
           const float lq = l[nt][x];
           const float inv = lq > 0.f ? 1.f / lq : 0.f;
           const int h = cur.g * G + q;

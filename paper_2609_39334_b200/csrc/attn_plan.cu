@@ -337,26 +337,7 @@ __device__ __forceinline__ void plan_emit_phase(const Params& P) {
     it.kv_end = max(0, min(L, it.limit0 + it.n_tok - 1));
     it.slot_off = -1;
     it.src0 = src_row + t * tpt;
-    {                                           // page segments of the chain, root first
-      int chain[SS_MAX_DEPTH];
-      int d = 0;
-      for (int a = it.node; a >= 0 && d < SS_MAX_DEPTH; a = P.node_parent[a]) chain[d++] = a;
-      int n_seg = 0, first = 0;
-      it.seg_first[0] = it.seg_first[1] = 0x7fffffff;
-      it.seg_off[0] = it.seg_off[1] = it.seg_off[2] = 0;
-      for (int c = d - 1; c >= 0; --c) {
-        const int n = chain[c];
-        const int np = (P.node_kv_len[n] + kPage - 1) / kPage;
-        if (np == 0) continue;
-        if (n_seg < kItemSegs) {
-          it.seg_off[n_seg] = static_cast<int32_t>(P.node_page_offsets[n]);
-          if (n_seg > 0) it.seg_first[n_seg - 1] = first;
-        }
-        first += np;
-        ++n_seg;
-      }
-      it.n_seg = n_seg <= kItemSegs ? n_seg : -1;
-    }
+    it.pad = 0;
     P.tile_items[n_stacked + e] = it;
   }
 
@@ -388,10 +369,7 @@ __device__ __forceinline__ void plan_emit_phase(const Params& P) {
     it.limit0 = it.kv_end;
     it.slot_off = P.node_level_off[n] + split;
     it.src0 = 0;
-    it.n_seg = 1;
-    it.seg_first[0] = it.seg_first[1] = 0x7fffffff;
-    it.seg_off[0] = static_cast<int32_t>(P.node_page_offsets[n]);
-    it.seg_off[1] = it.seg_off[2] = 0;
+    it.pad = 0;
     P.tile_items[e] = it;
   }
 }

@@ -27,7 +27,7 @@ constexpr int kMinSplitLen = 512;       // a split is at least this many keys
 enum PathClass : int32_t { kClassDecode = 0, kClassChain = 1, kClassGeneric = 2 };
 enum ItemKind : int32_t { kItemStacked = 0, kItemChain = 1 };
 
-// One tile of stacked query rows against a KV source.  64 bytes.
+// One tile of stacked query rows against a KV source.  40 bytes.
 struct alignas(8) TileItem {
   int32_t node;       // stacked: the shared node; chain: the path's leaf node
   int32_t tok0;       // stacked: index into dec_tok[]; chain: first query row (global token index)
@@ -38,15 +38,8 @@ struct alignas(8) TileItem {
   int32_t limit0;     // keys visible to the tile's first token; token i sees limit0 + i * (kind == chain)
   int32_t slot_off;   // stacked: partial slot relative to the token's slot base; chain: -1 (final output)
   int32_t src0;       // chain: row of q holding the tile's first token (stacked: rows come from dec_src[])
-  // The page segments of the source, so that the kernel need not walk the tree: segment d covers the virtual pages
-  // [seg_first[d], seg_first[d + 1]) of the key sequence (seg_first[0] = 0) and starts at node_pages[seg_off[d]].
-  // A stacked item has one segment (its node); a chain item one per non-empty node root -> leaf.  n_seg = -1: more
-  // than kItemSegs segments, the kernel walks the chain itself.
-  int32_t n_seg;
-  int32_t seg_first[2];   // of segments 1 and 2
-  int32_t seg_off[3];
+  int32_t pad;
 };
-constexpr int kItemSegs = 3;
 
 // One chunk of a decode path's private leaf.  32 bytes.
 struct alignas(16) LeafItem {

@@ -32,7 +32,8 @@ __device__ __forceinline__ void row_visit_node(RowState& r, const Params& P, int
   if (t1 <= t0) return;
   const int64_t pg0 = P.node_page_offsets[node];
   for (int t = t0; t < t1; ++t) {
-    const int64_t page = P.node_pages[pg0 + t / kPage];
+    int64_t page = P.node_pages[pg0 + t / kPage];
+    SS_CHECK_OR(page >= 0 && page < P.num_pages, &P.hdr->status, page = 0);
     const int64_t off = page * P.page_stride + static_cast<int64_t>(g) * P.head_stride +
                         static_cast<int64_t>(t % kPage) * P.token_stride + 4 * lane;
     float k[4], v[4];
@@ -111,6 +112,8 @@ __device__ __forceinline__ void tile_item_rows_exact(const Params& P, const Tile
 // moments ago.
 __device__ __forceinline__ void merge_row(const Params& P, int d, int h, int lane) {
   const int s0 = P.dec_slot_base[d], s1 = P.dec_slot_base[d + 1];
+  SS_CHECK_OR(s0 >= 0 && s0 <= s1 && s1 <= P.caps.slots && P.dec_tok[d] >= 0 && P.dec_tok[d] < P.total_q, &P.hdr->status,
+              return);
   float m = -INFINITY;
   for (int s = s0 + lane; s < s1; s += 32) m = fmaxf(m, __ldcg(P.part_lse + static_cast<int64_t>(s) * P.Hq + h));
   m = warp_max(m);
@@ -135,7 +138,9 @@ __device__ __forceinline__ void merge_row(const Params& P, int d, int h, int lan
 // are independent, so their loads are issued together: merging them one after another costs two memory round trips
 // per row, which is what a leaf item's last warp would otherwise wait for.
 __device__ __forceinline__ void merge_rows8(const Params& P, int d, int h0, int n_rows, int lane) {
-  const int s0 = P.dec_slot_base[d], s1 = P.dec_slot_base[d + 1];
+  int s0 = P.dec_slot_base[d], s1 = P.dec_slot_base[d + 1];
+  SS_CHECK_OR(s0 >= 0 && s0 <= s1 && s1 <= P.caps.slots && P.dec_tok[d] >= 0 && P.dec_tok[d] < P.total_q, &P.hdr->status,
+              return);
   float m[8];
 #pragma unroll
   for (int r = 0; r < 8; ++r) {

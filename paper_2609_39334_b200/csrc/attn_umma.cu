@@ -253,6 +253,9 @@ tile_items_umma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_
         const float lse = l > 0.f ? m * P.scale + __logf(l) : -INFINITY;
         const bool final_out = it.slot_off < 0;
         const int64_t slot = final_out ? 0 : static_cast<int64_t>(row_valid ? P.dec_slot_base[dec] : 0) + it.slot_off;
+        bool store_ok = true;
+        SS_CHECK_OR(!row_valid || (final_out ? (q_row >= 0 && q_row < P.total_q) : (slot >= 0 && slot < P.caps.slots)),
+                    &P.hdr->status, store_ok = false);
 #pragma unroll
         for (int c0 = 0; c0 < kHeadDim; c0 += 32) {
           uint32_t orow[32];
@@ -264,7 +267,7 @@ tile_items_umma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_
 #pragma unroll
             for (int x = 0; x < 32; ++x) orow[x] = 0u;
           }
-          if (!row_valid) continue;
+          if (!row_valid || !store_ok) continue;
           if (final_out) {
             uint4* dst = reinterpret_cast<uint4*>(P.out + (q_row * P.Hq + h) * kHeadDim + c0);
 #pragma unroll
@@ -286,7 +289,7 @@ tile_items_umma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_
                                    __uint_as_float(orow[4 * x + 2]) * inv, __uint_as_float(orow[4 * x + 3]) * inv);
           }
         }
-        if (row_valid) {
+        if (row_valid && store_ok) {
           if (final_out) { if (P.lse) P.lse[q_row * P.Hq + h] = lse; }
           else P.part_lse[slot * P.Hq + h] = lse;
         }
@@ -330,7 +333,8 @@ tile_items_umma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_
           const int vp = pos0 / kPage + lane;
           int d = 0;
           while (d + 1 < n_seg && vp >= C.seg_first_page[d + 1]) ++d;
-          const int64_t phys = P.node_pages[C.seg_page_off[d] + (vp - C.seg_first_page[d])];
+          int64_t phys = P.node_pages[C.seg_page_off[d] + (vp - C.seg_first_page[d])];
+          SS_CHECK_OR(phys >= 0 && phys < P.num_pages, &P.hdr->status, phys = 0);
           return static_cast<int>((phys * P.page_stride + static_cast<int64_t>(it.g) * P.head_stride) >> 7);
         };
         int next_coord = page_coord(0);

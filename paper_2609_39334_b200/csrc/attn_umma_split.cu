@@ -57,6 +57,7 @@ constexpr int kOffQ = 0;                       // 2 buffers (this item / next it
 constexpr int kOffK = 65536;
 constexpr int kOffV = kOffK + kStagesK * kStageBytes;
 constexpr int kUmmaSmem = kOffV + kStagesV * kStageBytes;   // + the control block in static shared memory
+static_assert(kColO + kHeadDim <= kTmemCols && kColS + kRing * kTile <= kColO, "score buffers and accumulator inside the allocated TMEM columns");
 
 struct Ctrl {
   // All per-buffer barriers are indexed by tile number modulo the ring / stage count and waited with the parity of
@@ -209,6 +210,7 @@ tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const _
       const bool row_valid = i < v.n_tok;
       int64_t q_src = 0;
       if (row_valid) q_src = P.dec_src[v.tok0 + i];
+      SS_CHECK_OR(q_src >= 0 && q_src < (P.q_src_offsets ? P.q_src_rows : P.total_q), &P.hdr->status, q_src = 0);
       const char* src = reinterpret_cast<const char*>(P.q + (q_src * P.Hq + (v.g * G + hl)) * kHeadDim);
       const uint32_t n_src = row_valid ? 16u : 0u;               // 0 source bytes: the 16 destination bytes are zeroed
 #pragma unroll
@@ -436,6 +438,14 @@ tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const _
       const float l_all = l + __uint_as_float(C.xmax[0][hf ^ 1][row]);
       pair_barrier();
       C.xmax[0][hf][row] = 0u;
+#ifdef SS_CHECKED
+      {                                                           // (warp-uniform outcome: the loads below are collective)
+        const bool in_range = !row_valid || (it.slot_off < 0 ? (q_row >= 0 && q_row < P.total_q)
+                                                             : (static_cast<int64_t>(P.dec_slot_base[dec]) + it.slot_off < P.caps.slots));
+        if (!in_range) set_status(&P.hdr->status, SS_ERR_BAD_INPUT);
+        if (!__all_sync(0xffffffffu, in_range)) ok = false;
+      }
+#endif
       if (ok) {
         const float inv = l_all > 0.f ? 1.f / l_all : 0.f;
         const float lse = l_all > 0.f ? m * P.scale + __logf(l_all) : -INFINITY;
@@ -532,7 +542,8 @@ tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const _
           const int vp = pos0 / kPage + pg;
           int d = 0;
           while (d + 1 < n_seg && vp >= seg_first[d + 1]) ++d;
-          const int64_t phys = P.node_pages[seg_off[d] + (vp - seg_first[d])];
+          int64_t phys = P.node_pages[seg_off[d] + (vp - seg_first[d])];
+          SS_CHECK_OR(phys >= 0 && phys < P.num_pages, &P.hdr->status, phys = 0);
           return static_cast<int>((phys * P.page_stride + static_cast<int64_t>(v.g) * P.head_stride) >> 7);
         };
         bool ok = true;

@@ -94,6 +94,22 @@ __device__ __forceinline__ float warp_max(float v) {
 }
 // First error wins: the status word keeps the first non-zero code written to it.
 __device__ __forceinline__ void set_status(int32_t* status, int32_t code) { atomicCAS(status, 0, code); }
+
+// Checked build (-DSS_CHECKED, libspecscale_checked.so): range predicates on the kernels' OWN address arithmetic - page
+// ids against the pool, partial slots against the workspace capacity, query / output rows against the tensors.  A
+// failed predicate records SS_ERR_BAD_INPUT in the status word and runs `fallback` (clamp the index or skip the
+// access), so nothing is ever accessed out of range.  In the production build the macro expands to nothing.
+#ifdef SS_CHECKED
+#define SS_CHECK_OR(cond, status_ptr, fallback)                         \
+  do {                                                                  \
+    if (!(cond)) {                                                      \
+      ::ss::set_status((status_ptr), SS_ERR_BAD_INPUT);                 \
+      fallback;                                                         \
+    }                                                                   \
+  } while (0)
+#else
+#define SS_CHECK_OR(cond, status_ptr, fallback) do { } while (0)
+#endif
 #endif
 
 }  // namespace ss

@@ -4,10 +4,105 @@
 // ss_topk_prune, asynchronous copies of every result back - all on the caller's stream, without a host
 // synchronisation, so that a caller that alternates between a few arenas and streams overlaps one step's copies
 // with another step's kernels.
+//
+// Rows nobody reads do not cross the bus: a duplicate candidate gets no forward pass (paper, Section "Computation
+// Deduplication"), so it has no query and no output of its own.  When the caller's q / out / lse buffers are
+// page-locked AND mapped (cudaHostAlloc / cudaHostRegister memory: the device can address them), the token ids go
+// first, the paths are deduplicated, and only then two small copy kernels move the query rows of the UNIQUE paths in
+// (read straight from the host buffer) and, after the attention, the live rows of out / lse back (written straight
+// into the host buffer) - how many rows those are is only known on the device, which is why kernels do it and not
+// cudaMemcpyAsync.  The copy kernels are a few persistent blocks, and the attention call is told to leave as many
+// SMs free (ss_attn_desc_t::max_sms): its tile and leaf blocks need an SM to themselves, and would otherwise wait
+// for a copy block that runs for as long as the bus takes.  Buffers that are not mapped take the plain path: every
+// logical candidate's rows are copied with cudaMemcpyAsync.
 #include "common.cuh"
 
 namespace ss {
 namespace host_step {
+
+constexpr int kCopyBlocks = 8;       // persistent blocks per copy kernel
+constexpr int kCopyThreads = 512;
+constexpr int kGatherBatch = 128;    // paths whose descriptors a block stages at a time
+
+// Query rows of the live unique paths, host -> device: path u's rows [u_q_src[u], + T) of the caller's buffer become
+// rows [u_q_offsets[u], + T) of the compact device buffer (a path's rows are contiguous on both sides; a batch of
+// consecutive paths is contiguous on the device side).  16-byte chunks, several in flight per thread.
+__global__ void __launch_bounds__(kCopyThreads)
+gather_q_from_host_kernel(const uint4* __restrict__ q_host, uint4* __restrict__ q_dev, const int32_t* __restrict__ num_unique,
+                          int32_t n_paths, const int64_t* __restrict__ u_q_offsets, const int64_t* __restrict__ u_q_src,
+                          int64_t row_chunks, int32_t* __restrict__ batch_counter) {
+  ss::grid_dependency_enter();
+  __shared__ int64_t s_off[kGatherBatch + 1], s_src[kGatherBatch];
+  __shared__ int s_batch;
+  int live = *num_unique;
+  live = live < 0 ? 0 : (live > n_paths ? n_paths : live);
+  for (;;) {
+    __syncthreads();
+    if (threadIdx.x == 0) s_batch = atomicAdd(batch_counter, 1);
+    __syncthreads();
+    const int p0 = s_batch * kGatherBatch;
+    if (p0 >= live) break;
+    const int np = min(kGatherBatch, live - p0);
+    for (int i = threadIdx.x; i <= np; i += blockDim.x) {
+      s_off[i] = u_q_offsets[p0 + i];
+      if (i < np) s_src[i] = u_q_src[p0 + i];
+    }
+    __syncthreads();
+    const int64_t row0 = s_off[0];
+    const int64_t n_chunks = (s_off[np] - row0) * row_chunks;
+    uint4* dst = q_dev + row0 * row_chunks;
+    for (int64_t c0 = threadIdx.x; c0 < n_chunks; c0 += 4LL * blockDim.x) {
+      uint4 v[4];
+#pragma unroll
+      for (int x = 0; x < 4; ++x) {
+        const int64_t c = c0 + static_cast<int64_t>(x) * blockDim.x;
+        if (c >= n_chunks) break;
+        const int64_t row = row0 + c / row_chunks;
+        int lo = 0, hi = np;                               // path of the batch that owns the row
+        while (hi - lo > 1) {
+          const int mid = (lo + hi) >> 1;
+          if (s_off[mid] <= row) lo = mid; else hi = mid;
+        }
+        v[x] = q_host[(s_src[lo] + (row - s_off[lo])) * row_chunks + c % row_chunks];
+      }
+#pragma unroll
+      for (int x = 0; x < 4; ++x) {
+        const int64_t c = c0 + static_cast<int64_t>(x) * blockDim.x;
+        if (c < n_chunks) dst[c] = v[x];
+      }
+    }
+  }
+}
+
+// The live rows of out / lse, device -> host: rows [0, u_q_offsets[U]) of the compact device buffers.
+__global__ void __launch_bounds__(kCopyThreads)
+rows_to_host_kernel(const uint4* __restrict__ out_dev, uint4* __restrict__ out_host, const uint4* __restrict__ lse_dev,
+                    uint4* __restrict__ lse_host, const int32_t* __restrict__ num_unique, int32_t n_paths,
+                    const int64_t* __restrict__ u_q_offsets, int64_t out_row_chunks, int64_t lse_row_bytes) {
+  ss::grid_dependency_enter();
+  int live = *num_unique;
+  live = live < 0 ? 0 : (live > n_paths ? n_paths : live);
+  const int64_t rows = u_q_offsets[live];
+  const int64_t tid = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  const int64_t nt = static_cast<int64_t>(gridDim.x) * blockDim.x;
+  const int64_t n_out = rows * out_row_chunks;
+  for (int64_t c0 = tid; c0 < n_out; c0 += 4 * nt) {
+    uint4 v[4];
+#pragma unroll
+    for (int x = 0; x < 4; ++x)
+      if (c0 + x * nt < n_out) v[x] = out_dev[c0 + x * nt];
+#pragma unroll
+    for (int x = 0; x < 4; ++x)
+      if (c0 + x * nt < n_out) out_host[c0 + x * nt] = v[x];
+  }
+  if (lse_host) {
+    const int64_t n_bytes = rows * lse_row_bytes, n_lse = n_bytes / 16;
+    for (int64_t c = tid; c < n_lse; c += nt) lse_host[c] = lse_dev[c];
+    const float* tail_src = reinterpret_cast<const float*>(lse_dev + n_lse);       // (< 16 bytes)
+    float* tail_dst = reinterpret_cast<float*>(lse_host + n_lse);
+    if (tid < (n_bytes - n_lse * 16) / 4) tail_dst[tid] = tail_src[tid];
+  }
+}
 
 struct Arena {                       // device-side layout of one step
   // staged inputs
@@ -19,6 +114,7 @@ struct Arena {                       // device-side layout of one step
   int32_t* num_unique;
   int32_t* u_leaf; int32_t* u_q_len; int64_t* u_q_offsets; int64_t* u_q_src;
   void* out; float* lse; int32_t* survivors; uint8_t* keep;
+  int32_t* copy_counter;             // batch counter of the query gather (zeroed every step)
   // workspaces of the three calls
   void* dedup_ws; size_t dedup_ws_bytes;
   void* attn_ws; size_t attn_ws_bytes;
@@ -29,7 +125,9 @@ struct Arena {                       // device-side layout of one step
 static size_t at_least_one(int64_t n) { return static_cast<size_t>(n > 0 ? n : 1); }
 
 // The attention descriptor of this step: the caller's resident fields + the staged per-path arrays.
-static ss_attn_desc_t step_desc(const ss_host_step_t& s, const Arena& a) {
+// `compact_q`: the device buffer holds the unique paths' rows at u_q_offsets (gathered from the host); otherwise it
+// holds every logical candidate's rows and the attention reads them in place through u_q_src.
+static ss_attn_desc_t step_desc(const ss_host_step_t& s, const Arena& a, bool compact_q = false, int max_sms = 0) {
   ss_attn_desc_t d = *s.attn;
   d.num_paths = s.n_paths;
   d.num_paths_dev = a.num_unique;
@@ -37,8 +135,9 @@ static ss_attn_desc_t step_desc(const ss_host_step_t& s, const Arena& a) {
   d.path_q_len = a.u_q_len;
   d.q_offsets = a.u_q_offsets;
   d.total_q = s.total_q;
-  d.q_src_offsets = a.u_q_src;
-  d.q_src_rows = s.total_q;
+  d.q_src_offsets = compact_q ? nullptr : a.u_q_src;
+  d.q_src_rows = compact_q ? 0 : s.total_q;
+  d.max_sms = max_sms;
   d.q = a.q;
   d.out = a.out;
   d.lse = a.lse;
@@ -73,6 +172,7 @@ static int32_t carve(const ss_host_step_t& s, void* base, Arena* a) {
   a->lse = c.take<float>(at_least_one(s.total_q) * static_cast<size_t>(s.attn->num_q_heads));
   a->survivors = c.take<int32_t>(P * static_cast<size_t>(s.top_k));
   a->keep = c.take<uint8_t>(N);
+  a->copy_counter = c.take<int32_t>(4);
   int32_t rc = ss_dedup_workspace_bytes(s.n_paths, &a->dedup_ws_bytes);
   if (rc != SS_OK) return rc;
   a->dedup_ws = c.take<char>(a->dedup_ws_bytes);
@@ -154,7 +254,29 @@ extern "C" int32_t ss_candidate_step_host(const ss_host_step_t* step, void* devi
   SS_COPY(a.path_leaf_node, s.path_leaf_node, N * 4, H2D);
   SS_COPY(a.path_q_len, s.path_q_len, N * 4, H2D);
   SS_COPY(a.q_offsets, s.q_offsets, (N + 1) * 8, H2D);
-  SS_COPY(a.q, s.q, q_bytes, H2D);
+  // mapped q / out / lse: only the unique paths' rows cross the bus (see the top of the file)
+  void *q_map = nullptr, *out_map = nullptr, *lse_map = nullptr;
+  bool slim = s.total_q > 0 && s.n_paths > 0 && row * sizeof(__nv_bfloat16) % 16 == 0;
+  if (slim && (cudaHostGetDevicePointer(&q_map, const_cast<void*>(s.q), 0) != cudaSuccess ||
+               cudaHostGetDevicePointer(&out_map, s.out, 0) != cudaSuccess ||
+               (s.lse && cudaHostGetDevicePointer(&lse_map, s.lse, 0) != cudaSuccess))) {
+    (void)cudaGetLastError();
+    slim = false;
+  }
+  int dev_sms = 0;
+  if (slim) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&dev_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        dev_sms <= 4 * kCopyBlocks) {
+      (void)cudaGetLastError();
+      slim = false;
+    }
+  }
+  if (slim) {
+    if (cudaMemsetAsync(a.copy_counter, 0, 16, st) != cudaSuccess) { (void)cudaGetLastError(); return SS_ERR_CUDA; }
+  } else {
+    SS_COPY(a.q, s.q, q_bytes, H2D);
+  }
   SS_COPY(a.scores, s.scores, N * 4, H2D);
   SS_COPY(a.seg_offsets, s.seg_offsets, (P + 1) * 4, H2D);
 
@@ -166,7 +288,13 @@ extern "C" int32_t ss_candidate_step_host(const ss_host_step_t* step, void* devi
   rc = ss_gather_unique_paths(a.unique_paths, a.num_unique, s.n_paths, a.path_leaf_node, a.path_q_len, a.q_offsets,
                               a.u_leaf, a.u_q_len, a.u_q_offsets, a.u_q_src, stream);
   if (rc != SS_OK) return rc;
-  const ss_attn_desc_t d = step_desc(s, a);
+  const int64_t row_chunks = static_cast<int64_t>(row * sizeof(__nv_bfloat16) / 16);
+  if (slim)
+    SS_LAUNCH(gather_q_from_host_kernel, kCopyBlocks, kCopyThreads, 0, st, static_cast<const uint4*>(q_map),
+              static_cast<uint4*>(a.q), static_cast<const int32_t*>(a.num_unique), s.n_paths,
+              static_cast<const int64_t*>(a.u_q_offsets), static_cast<const int64_t*>(a.u_q_src), row_chunks, a.copy_counter);
+  // (two copy kernels of other steps may be running beside this step's attention: their SMs are left alone)
+  const ss_attn_desc_t d = step_desc(s, a, slim, slim ? dev_sms - 2 * kCopyBlocks : 0);
   rc = ss_tree_attention(&d, a.attn_ws, a.attn_ws_bytes, stream);
   if (rc != SS_OK) return rc;
   rc = ss_topk_prune(a.scores, a.seg_offsets, s.n_segments, s.n_paths, s.top_k, a.survivors, a.keep, a.topk_ws,
@@ -181,8 +309,15 @@ extern "C" int32_t ss_candidate_step_host(const ss_host_step_t* step, void* devi
   if (s.slot_out) SS_COPY(s.slot_out, a.slot_out, N * 4, D2H);
   SS_COPY(s.num_unique, a.num_unique, 4, D2H);
   SS_COPY(s.u_q_offsets, a.u_q_offsets, (N + 1) * 8, D2H);
-  SS_COPY(s.out, a.out, q_bytes, D2H);
-  if (s.lse) SS_COPY(s.lse, a.lse, lse_bytes, D2H);
+  if (slim) {
+    SS_LAUNCH(rows_to_host_kernel, kCopyBlocks, kCopyThreads, 0, st, static_cast<const uint4*>(a.out),
+              static_cast<uint4*>(out_map), reinterpret_cast<const uint4*>(a.lse), static_cast<uint4*>(lse_map),
+              static_cast<const int32_t*>(a.num_unique), s.n_paths, static_cast<const int64_t*>(a.u_q_offsets), row_chunks,
+              static_cast<int64_t>(s.attn->num_q_heads) * 4);
+  } else {
+    SS_COPY(s.out, a.out, q_bytes, D2H);
+    if (s.lse) SS_COPY(s.lse, a.lse, lse_bytes, D2H);
+  }
   SS_COPY(s.survivors, a.survivors, P * static_cast<size_t>(s.top_k) * 4, D2H);
   SS_COPY(s.keep, a.keep, N, D2H);
   SS_COPY(s.device_status, a.attn_ws, sizeof(int32_t), D2H);     // first word of the attention workspace

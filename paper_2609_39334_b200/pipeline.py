@@ -182,6 +182,27 @@ class HostStepPipeline:
         self.h2d_bytes = sum(t.numel() * t.element_size() for t in self.sets[0]["h_in"].values())
         self.d2h_bytes = sum(t.numel() * t.element_size() for t in self.sets[0]["h_out"].values())
 
+    def measure_traffic(self):
+        """Runs one step on set 0 and sets h2d_bytes / d2h_bytes to what that step moved over the bus.  Page-locked
+        buffers from torch are mapped, so the call fetches only the unique paths' query rows and returns only the live
+        rows of out / lse; whether it did is read off a sentinel row past the live ones (left untouched if so)."""
+        s = self.sets[0]
+        o, i = s["h_out"], s["h_in"]
+        tq_all = o["out"].shape[0]
+        o["out"][tq_all - 1].fill_(-7.0)
+        self.submit(0)
+        s["stream"].synchronize()
+        U = int(o["num_unique"][0])
+        tq_live = int(o["u_q_offsets"][U]) if self.resident.N else 0
+        slim = tq_live < tq_all and bool((o["out"][tq_all - 1].float() == -7.0).all())
+        if slim:
+            row = o["out"].shape[1] * o["out"].shape[2] * 2
+            small_in = sum(t.numel() * t.element_size() for k, t in i.items() if k != "q")
+            small_out = sum(t.numel() * t.element_size() for k, t in o.items() if k not in ("out", "lse"))
+            self.h2d_bytes = small_in + tq_live * row
+            self.d2h_bytes = small_out + tq_live * (row + o["lse"].shape[1] * 4)
+        return slim
+
     def submit(self, i: int):
         s = self.sets[i % len(self.sets)]
         B.ss_candidate_step_host(s["step"], s["arena"], stream=s["stream"])

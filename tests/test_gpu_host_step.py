@@ -63,3 +63,24 @@ def test_host_step_empty_batch_and_errors():
     s["stream"].synchronize()
     assert int(s["h_out"]["num_unique"][0]) == 0 and int(s["h_out"]["u_q_offsets"][0]) == 0
     assert int(s["h_out"]["device_status"][0]) == B.SS_OK
+
+
+@pytest.mark.parametrize("cfg", [2, 4])
+def test_host_step_moves_only_unique_rows_when_the_buffers_are_mapped(cfg):
+    """Page-locked buffers are mapped into the device's address space: the call then fetches the query rows of the unique
+    paths only and returns only the live rows of out / lse (a duplicate gets no forward pass, hence no query and no
+    output of its own).  Rows past the live ones must stay as the caller left them."""
+    w = synth.make_config(cfg)
+    pipe = DevicePipeline(w, DEV)
+    pipe.step()
+    r_dev = pipe.results()
+    host = HostStepPipeline(pipe, depth=1)
+    full_in, full_out = host.h2d_bytes, host.d2h_bytes
+    assert host.measure_traffic()
+    U, tq = r_dev["num_unique"], r_dev["total_q"]
+    assert U < w.num_paths and tq < w.total_q
+    row = w.num_q_heads * w.head_dim * 2
+    assert host.h2d_bytes == full_in - (w.total_q - tq) * row
+    assert host.d2h_bytes == full_out - (w.total_q - tq) * (row + w.num_q_heads * 4)
+    r = host.results(0)
+    assert np.array_equal(r["out"], r_dev["out"]) and np.array_equal(r["lse"], r_dev["lse"])

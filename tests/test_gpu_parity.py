@@ -104,7 +104,7 @@ def check_attention(r, w, ref, max_paths=48, tight=True, host_w=None):
     return err.max(), err.mean(), lerr
 
 
-MODES = [("fast", 0), ("flow", B.SS_FLAG_TILES_FLOW), ("two_cta", B.SS_FLAG_TILES_2CTA), ("no_tcgen05", B.SS_FLAG_NO_TCGEN05),
+MODES = [("fast", 0), ("two_cta", B.SS_FLAG_TILES_2CTA), ("no_tcgen05", B.SS_FLAG_NO_TCGEN05),
          ("generic", B.SS_FLAG_FORCE_GENERIC)]
 
 
