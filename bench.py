@@ -630,7 +630,7 @@ def main():
     # ---- end to end: ss_candidate_step_host - inputs from pinned host memory, results back to the host, every step --
     if not args.no_e2e:
         from paper_2609_39334_b200.pipeline import HostStepPipeline
-        host = HostStepPipeline(pipe, depth=args.e2e_depth)
+        host = HostStepPipeline(pipe, depth=args.e2e_depth, compact=True)
         slim = host.measure_traffic()                     # (bytes per step as the call really moves them)
         for i in range(args.e2e_depth):
             host.submit(i)
@@ -655,10 +655,10 @@ def main():
                       "h2d_bytes_per_step": int(host.h2d_bytes), "d2h_bytes_per_step": int(host.d2h_bytes),
                       "ms_per_step": e2e_ms, "steps": n_e2e, "sets_in_flight": args.e2e_depth,
                       "api": "ss_candidate_step_host",
-                      "unique_rows_only": bool(slim),
+                      "live_rows_only_back": bool(slim),
                       "note": "KV pool stays resident (it is the cache); every step copies candidates and scores from "
-                              "pinned host memory, fetches the query rows of the unique paths from it after the "
-                              "deduplication and writes the live rows of out / lse and all other results back; steps "
+                              "pinned host memory, copies every candidate's query rows in and returns the live rows of out / lse "
+                              "(a small kernel writes them into the mapped host buffers) and all other results; steps "
                               "alternate between independent (host buffers, device arena, stream) sets so copies "
                               "overlap kernels"}
         del host

@@ -195,9 +195,10 @@ typedef struct ss_attn_desc {
   int32_t num_q_heads, num_kv_heads; /* Hq % Hkv == 0 */
   int32_t head_dim, page_size;       /* 128, 16 */
   float sm_scale;                    /* 0 => 1/sqrt(head_dim) */
-  int32_t max_sms;                   /* 0: use every SM; otherwise the attention kernels occupy at most this many
-                                        (their blocks need an SM to themselves: a caller that runs long-lived small
-                                        kernels beside the call - copy kernels - leaves those SMs out) */
+  int32_t max_sms;                   /* 0: use every SM; otherwise the tile and leaf kernels occupy at most this many.
+                                        Their blocks are persistent and need an SM to themselves, so other streams'
+                                        kernels wait for the whole call unless a few SMs are left out (the
+                                        host-buffer step does that for the copy kernel of the step before it) */
   const void* k_pool;                /* bf16 */
   const void* v_pool;                /* bf16 */
   int64_t num_pages;                 /* pages addressable through k_pool / v_pool */
@@ -254,7 +255,8 @@ int32_t ss_tree_attention(const ss_attn_desc_t* desc /* host */, void* workspace
  *                 fewer than k candidates
  *   keep_out      uint8 [n_total]        1 iff the candidate survives (entries outside every segment: 0)
  *   workspace     >= ss_topk_workspace_bytes(n_total) bytes, 256-byte aligned
- * Errors: SS_ERR_INVALID_ARG, SS_ERR_WORKSPACE_TOO_SMALL, SS_ERR_CUDA.
+ * Errors: SS_ERR_INVALID_ARG, SS_ERR_WORKSPACE_TOO_SMALL, SS_ERR_CUDA (host); SS_ERR_BAD_INPUT via
+ * ss_last_device_status(workspace) if a segment does not lie inside [0, n_total] (it is then treated as empty).
  * ======================================================================================================= */
 int32_t ss_topk_workspace_bytes(int32_t n_total, size_t* out_bytes /* host */);
 int32_t ss_topk_prune(const float* scores, const int32_t* seg_offsets, int32_t n_segments, int32_t n_total,
@@ -280,7 +282,8 @@ int32_t ss_topk_prune(const float* scores, const int32_t* seg_offsets, int32_t n
  *   final_out     uint8 [n_segments] 1 iff rule 2 fired or every candidate of the segment is verified (then
  *                 selected_out equals the survivors of ss_topk_prune)
  *   workspace     >= ss_topk_workspace_bytes(n_total) bytes, 256-byte aligned
- * Errors: SS_ERR_INVALID_ARG, SS_ERR_WORKSPACE_TOO_SMALL, SS_ERR_CUDA.
+ * Errors: SS_ERR_INVALID_ARG, SS_ERR_WORKSPACE_TOO_SMALL, SS_ERR_CUDA (host); SS_ERR_BAD_INPUT via
+ * ss_last_device_status(workspace) if a segment does not lie inside [0, n_total] (it is then treated as empty).
  * ======================================================================================================= */
 int32_t ss_early_prune(const float* scores, const uint8_t* verified, const int32_t* seg_offsets, int32_t n_segments,
                        int32_t n_total, int32_t k, uint8_t* pruned_out, int32_t* selected_out, uint8_t* final_out,
@@ -303,10 +306,10 @@ int32_t ss_early_prune(const float* scores, const uint8_t* verified, const int32
  *   draw_offsets  int64 [n_seq+1]       draws of sequence s are draw_offsets[s] .. draw_offsets[s+1]-1
  *                                       (draw_offsets[s+1] - draw_offsets[s] = its potential size)
  *   uniforms      fp32 [draw_offsets[n_seq]]  in [0, 1)
- *   n_seq, vocab  host;  temperature host > 0
+ *   n_seq, vocab  host;  temperature host > 0;  vocab <= 2097152 (else SS_ERR_UNSUPPORTED)
  *   tokens_out    int32 [draws]   sampled token of every draw
  *   seq_out       int64 [draws]   the sequence every draw belongs to
- * Errors: SS_ERR_INVALID_ARG, SS_ERR_CUDA.
+ * Errors: SS_ERR_INVALID_ARG, SS_ERR_UNSUPPORTED, SS_ERR_CUDA.
  * ======================================================================================================= */
 int32_t ss_branch_sample(const float* logits, const int64_t* draw_offsets, const float* uniforms, int32_t n_seq,
                          int32_t vocab, float temperature, int32_t* tokens_out, int64_t* seq_out, void* stream);
@@ -360,11 +363,11 @@ int32_t ss_build_prefix_tree(const int32_t* tok_ids, const int64_t* tok_offsets,
  *   asynchronous copies host -> device of every per-step input  ->  ss_dedup_paths  ->  ss_gather_unique_paths  ->
  *   ss_tree_attention (queries read in place through the gathered offsets)  ->  ss_topk_prune  ->
  *   asynchronous copies device -> host of every result.
- * If q, out and lse are page-locked AND mapped into the device's address space (memory from cudaHostAlloc or
- * cudaHostRegister), the rows of duplicate candidates never cross the bus: the queries are fetched after the
- * deduplication, for the unique paths only, by a small kernel that reads the host buffer directly, and only the
- * live rows of out / lse (the first u_q_offsets[num_unique]) are written back, again by a kernel; the rest of
- * out / lse is left untouched.  Buffers that are not mapped are copied whole with cudaMemcpyAsync.
+ * With SS_STEP_COMPACT_TRANSFERS in `flags`, and out / lse page-locked AND mapped into the device's address space
+ * (memory from cudaHostAlloc / cudaHostRegister), only the live rows of out / lse come back - the first
+ * u_q_offsets[num_unique]: a duplicate candidate gets no forward pass, hence no output of its own - written by a small
+ * kernel straight into the host buffers; the rest of out / lse is left untouched.  (Buffers the device cannot address
+ * are returned whole, as without the flag.)
  * Everything is enqueued on `stream`; the call does not synchronise, and it allocates nothing: staging buffers,
  * results and the workspaces of the three calls are carved out of `device_arena` (caller-owned, 256-byte aligned,
  * >= ss_candidate_step_host_arena_bytes).  The KV pool and the tree stay resident on the device: they are the
@@ -385,11 +388,13 @@ int32_t ss_build_prefix_tree(const int32_t* tok_ids, const int64_t* tok_offsets,
  * Errors: SS_ERR_INVALID_ARG, SS_ERR_WORKSPACE_TOO_SMALL, SS_ERR_UNSUPPORTED, SS_ERR_CUDA (host); the device-side
  * errors of ss_tree_attention arrive in *device_status.
  * ======================================================================================================= */
+#define SS_STEP_COMPACT_TRANSFERS 0x1u   /* return only the live rows of out / lse (needs them mapped, see above) */
 typedef struct ss_host_step {
   uint32_t struct_size;              /* = sizeof(ss_host_step_t) */
   uint32_t dedup_flags;              /* 0 or SS_FLAG_WEAK_HASH */
   const ss_attn_desc_t* attn;        /* host; resident fields only (see above) */
-  int32_t n_paths, n_segments, top_k, reserved0;
+  int32_t n_paths, n_segments, top_k;
+  uint32_t flags;                    /* 0 or SS_STEP_COMPACT_TRANSFERS */
   int64_t total_tok;                 /* = tok_offsets[n_paths] - tok_offsets[0], and tok_offsets[0] must be 0 */
   int64_t total_q;                   /* = q_offsets[n_paths], and q_offsets[0] must be 0 */
   /* per-step inputs, host memory */

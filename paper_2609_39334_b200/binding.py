@@ -30,6 +30,7 @@ SS_FLAG_NO_TCGEN05 = 0x4
 SS_FLAG_WEAK_HASH = 0x8
 SS_FLAG_TILES_2CTA = 0x10
 SS_MAX_DEPTH = 16
+SS_STEP_COMPACT_TRANSFERS = 0x1
 SS_DEDUP_STATIC_MAX_PATHS = 65536
 
 EXPORTS = [
@@ -201,7 +202,7 @@ class ss_host_step_t(ctypes.Structure):
         ("struct_size", ctypes.c_uint32), ("dedup_flags", ctypes.c_uint32),
         ("attn", ctypes.c_void_p),
         ("n_paths", ctypes.c_int32), ("n_segments", ctypes.c_int32), ("top_k", ctypes.c_int32),
-        ("reserved0", ctypes.c_int32),
+        ("flags", ctypes.c_uint32),
         ("total_tok", ctypes.c_int64), ("total_q", ctypes.c_int64),
     ] + [(n, ctypes.c_void_p) for n in (
         "tok_ids", "tok_offsets", "ctx_key", "slot_in", "path_leaf_node", "path_q_len", "q_offsets", "q", "scores",
@@ -216,12 +217,13 @@ HOST_STEP_RESULTS = ("canon", "path_to_unique", "unique_paths", "multiplicity", 
 
 
 def make_host_step(attn_desc: "ss_attn_desc_t", *, n_paths, n_segments, top_k, total_tok, total_q, host_in: dict,
-                   host_out: dict, dedup_flags=0) -> ss_host_step_t:
+                   host_out: dict, dedup_flags=0, flags=0) -> ss_host_step_t:
     """Fills ss_host_step_t from dictionaries of HOST tensors (page-locked for asynchronous copies) keyed by the field
     names.  The returned object keeps references to the descriptor and the tensors."""
     s = ss_host_step_t()
     s.struct_size = ctypes.sizeof(ss_host_step_t)
     s.dedup_flags = dedup_flags
+    s.flags = flags
     s.attn = ctypes.addressof(attn_desc)
     s.n_paths, s.n_segments, s.top_k = int(n_paths), int(n_segments), int(top_k)
     s.total_tok, s.total_q = int(total_tok), int(total_q)

@@ -4,7 +4,7 @@
 #include "common.cuh"
 
 namespace ss {
-long long g_launch_count = 0;
+std::atomic<long long> g_launch_count{0};
 
 bool pdl_enabled() {
   static const bool on = std::getenv("SS_NO_PDL") == nullptr;
@@ -39,4 +39,4 @@ extern "C" int32_t ss_last_device_status(const void* workspace, void* stream, in
   return SS_OK;
 }
 
-extern "C" int64_t ss_launch_count(void) { return ss::g_launch_count; }
+extern "C" int64_t ss_launch_count(void) { return ss::g_launch_count.load(std::memory_order_relaxed); }

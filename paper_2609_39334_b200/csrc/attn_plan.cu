@@ -23,7 +23,7 @@ constexpr int kGridThreads = 256;
 
 // In-place exclusive scan of a[0..n) by one whole block: every thread sums a contiguous chunk, the chunk sums are
 // scanned across the block, then every thread rewrites its chunk.  Returns the total to every thread.
-__device__ int block_excl_scan(int32_t* a, int n) {
+__device__ int block_excl_scan_chunks(int32_t* a, int n) {
   __shared__ int warp_tot[32];
   __shared__ int total_s;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
@@ -59,6 +59,20 @@ __device__ int block_excl_scan(int32_t* a, int n) {
   }
   __syncthreads();
   return total_s;
+}
+
+// The same scan for an array in GLOBAL memory: it goes through the block's staging buffer in shared memory when it
+// fits (coalesced in, scanned on chip, coalesced out) - every thread walking its own contiguous chunk of a global
+// array makes each load touch 32 different sectors, which cost the one-block scan kernel most of its time.
+constexpr int kScanStage = 16384;                  // entries of the staging buffer (64 KB, dynamic shared memory)
+__device__ int block_excl_scan(int32_t* a, int n, int32_t* stage) {
+  if (stage == nullptr || n > kScanStage) return block_excl_scan_chunks(a, n);
+  __syncthreads();
+  for (int i = threadIdx.x; i < n; i += blockDim.x) stage[i] = a[i];
+  const int total = block_excl_scan_chunks(stage, n);      // (starts and ends with a barrier)
+  for (int i = threadIdx.x; i < n; i += blockDim.x) a[i] = stage[i];
+  __syncthreads();
+  return total;
 }
 
 // Block-uniform read of the status word (every thread gets the same answer, so an early return cannot leave
@@ -162,7 +176,8 @@ __device__ __forceinline__ void plan_paths_phase(const Params& P) {
 }
 
 // ---- every prefix sum -------------------------------------------------------------------------------------------------
-__device__ __forceinline__ void plan_scan_phase(const Params& P) {   // one whole block; block-uniform returns only
+__device__ __forceinline__ void plan_scan_phase(const Params& P, int32_t* stage) {   // one whole block; block-uniform
+                                                                                     // returns only; stage: see block_excl_scan
   __shared__ int s_total_tiles;
   PlanHeader* hdr = P.hdr;
   if (block_failed(hdr)) return;
@@ -174,7 +189,7 @@ __device__ __forceinline__ void plan_scan_phase(const Params& P) {   // one whol
 
   // decode ranks
   for (int p = tid; p < live; p += nt) P.path_dec_rank[p] = (P.path_class[p] == kClassDecode) ? 1 : 0;
-  const int n_dec = block_excl_scan(P.path_dec_rank, live);
+  const int n_dec = block_excl_scan(P.path_dec_rank, live, stage);
   if (tid == 0) {
     P.path_dec_rank[live] = n_dec;
     hdr->n_dec = n_dec;
@@ -228,7 +243,7 @@ __device__ __forceinline__ void plan_scan_phase(const Params& P) {   // one whol
     for (int a = P.node_parent[n]; a >= 0; a = P.node_parent[a]) off += P.node_own_slots[a];
     P.node_level_off[n] = off;
   }
-  const int n_stacked = block_excl_scan(P.node_item_base, N);
+  const int n_stacked = block_excl_scan(P.node_item_base, N, stage);
   if (tid == 0) P.node_item_base[N] = n_stacked;
 
   // decode paths: partial slots, leaf items; chain paths: tile items
@@ -247,9 +262,9 @@ __device__ __forceinline__ void plan_scan_phase(const Params& P) {   // one whol
     P.path_leaf_base[p] = leaf_items;
     P.path_chain_base[p] = chain_items;
   }
-  const int n_slots = block_excl_scan(P.path_slot_base, live);
-  const int n_leaf_items = block_excl_scan(P.path_leaf_base, live);
-  const int n_chain = block_excl_scan(P.path_chain_base, live);
+  const int n_slots = block_excl_scan(P.path_slot_base, live, stage);
+  const int n_leaf_items = block_excl_scan(P.path_leaf_base, live, stage);
+  const int n_chain = block_excl_scan(P.path_chain_base, live, stage);
   if (tid == 0) {
     hdr->n_slots = n_slots;
     hdr->n_stacked_items = n_stacked;
@@ -386,7 +401,8 @@ __global__ void __launch_bounds__(kGridThreads) plan_paths_kernel(const Params P
 }
 __global__ void __launch_bounds__(kScanThreads) plan_scan_kernel(const Params P) {
   ss::grid_dependency_enter();
-  plan_scan_phase(P);
+  extern __shared__ __align__(16) int32_t scan_stage[];
+  plan_scan_phase(P, scan_stage);
 }
 __global__ void __launch_bounds__(kGridThreads) plan_emit_kernel(const Params P) {
   ss::grid_dependency_enter();
@@ -448,7 +464,7 @@ __global__ void __launch_bounds__(kScanThreads) plan_small_kernel(const Params P
   if (!failed) {
     plan_paths_phase(P);
     __syncthreads();
-    plan_scan_phase(P);
+    plan_scan_phase(P, nullptr);                     // (the arrays are in shared memory already)
     failed = block_failed(P.hdr);
   }
   if (!failed) {
@@ -488,7 +504,18 @@ int32_t launch_plan(const Params& P, cudaStream_t st) {
   if (blocks > 1184) blocks = 1184;
   SS_LAUNCH(plan_nodes_kernel, blocks, kGridThreads, 0, st, P);
   SS_LAUNCH(plan_paths_kernel, blocks, kGridThreads, 0, st, P);
-  SS_LAUNCH(plan_scan_kernel, 1, kScanThreads, 0, st, P);
+  {
+    static bool configured[kDeviceSlots] = {false};
+    const int dev_slot = current_device_slot();
+    if (dev_slot < 0 || !configured[dev_slot]) {
+      if (cudaFuncSetAttribute(plan_scan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanStage * 4) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return SS_ERR_CUDA;
+      }
+      if (dev_slot >= 0) configured[dev_slot] = true;
+    }
+  }
+  SS_LAUNCH(plan_scan_kernel, 1, kScanThreads, kScanStage * 4, st, P);
   SS_LAUNCH(plan_emit_kernel, blocks, kGridThreads, 0, st, P);
   return SS_OK;
 }

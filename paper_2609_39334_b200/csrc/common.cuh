@@ -3,6 +3,7 @@
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
 #include <stdint.h>
+#include <atomic>
 #include <stddef.h>
 
 #include "../../include/specscale.h"
@@ -10,7 +11,7 @@
 namespace ss {
 
 // Host-side count of kernel launches made by this library (diagnostic, see ss_launch_count).
-extern long long g_launch_count;
+extern std::atomic<long long> g_launch_count;   // (atomic: hosts may call from one thread per stream)
 
 inline cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
 
@@ -36,7 +37,7 @@ bool pdl_enabled();
     ss_cfg_.attrs = ss_attr_;                                                     \
     ss_cfg_.numAttrs = ::ss::pdl_enabled() ? 1 : 0;                               \
     const cudaError_t ss_err_ = cudaLaunchKernelEx(&ss_cfg_, kernel, __VA_ARGS__); \
-    ++::ss::g_launch_count;                                                       \
+    ::ss::g_launch_count.fetch_add(1, std::memory_order_relaxed);                 \
     if (ss_err_ != cudaSuccess || cudaPeekAtLastError() != cudaSuccess) {         \
       (void)cudaGetLastError();                                                   \
       return SS_ERR_CUDA;                                                         \

@@ -298,6 +298,63 @@ __device__ __forceinline__ bool last_block_arrives(unsigned int* counter) {
   return s_last;
 }
 
+// Sort by counting, for batches too large for one block's shared-memory sort and too small to be worth a radix sort's
+// twelve launches: the rank of a path is the number of paths with a smaller (sort key, index) pair, counted by brute
+// force - n^2 comparisons, 0.27 G at 16384 paths, spread over the whole device (a few microseconds), against a
+// bitonic sort by a single block (~0.25 ms there: one SM, a hundred barrier-separated stages).  One thread per path;
+// the keys go through shared memory in tiles.
+constexpr int kRankThreads = 256;
+constexpr int kRankTile = 2048;
+constexpr int kRankSortMax = 32768;
+
+// Block (bi, bj) counts, for the 256 paths of group bi, the smaller pairs among the 2048 paths of tile bj and adds
+// the counts to rank_acc[] (zeroed before the launch); the block that completes a group - the last of its tiles to
+// arrive at group_done[bi] - scatters the group's keys and indices to their ranks.
+__global__ void __launch_bounds__(kRankThreads)
+rank_sort_kernel(const uint32_t* __restrict__ keys_in, int n, int n_tiles, int* rank_acc, unsigned int* group_done,
+                 uint32_t* __restrict__ keys_out, uint32_t* __restrict__ idx_out) {
+  ss::grid_dependency_enter();
+  __shared__ __align__(16) uint32_t tile[kRankTile];
+  __shared__ bool s_last;
+  const int bi = blockIdx.x / n_tiles, bj = blockIdx.x - bi * n_tiles;
+  const int i = bi * kRankThreads + threadIdx.x;
+  const uint32_t k = i < n ? keys_in[i] : 0xffffffffu;
+  const int base = bj * kRankTile;
+  for (int t = threadIdx.x; t < kRankTile; t += kRankThreads) tile[t] = base + t < n ? keys_in[base + t] : 0xffffffffu;
+  __syncthreads();
+  int cnt = 0;
+  // paths before this one count when their key is <= k, paths after it when it is < k (ties go by index); a tile
+  // that lies wholly on one side of the group's own paths takes the cheap uniform loop
+  if (base + kRankTile <= bi * kRankThreads) {
+#pragma unroll 4
+    for (int t = 0; t < kRankTile; t += 4) {
+      const uint4 v = *reinterpret_cast<const uint4*>(&tile[t]);
+      cnt += (v.x <= k) + (v.y <= k) + (v.z <= k) + (v.w <= k);
+    }
+  } else if (base >= (bi + 1) * kRankThreads) {
+#pragma unroll 4
+    for (int t = 0; t < kRankTile; t += 4) {         // (padding entries are 0xffffffff: never < k)
+      const uint4 v = *reinterpret_cast<const uint4*>(&tile[t]);
+      cnt += (v.x < k) + (v.y < k) + (v.z < k) + (v.w < k);
+    }
+  } else {
+    const int n_here = min(kRankTile, n - base);
+    for (int t = 0; t < n_here; ++t) cnt += (tile[t] < k) || (tile[t] == k && base + t < i);
+  }
+  if (i < n && cnt) atomicAdd(&rank_acc[i], cnt);
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) s_last = atomicAdd(&group_done[bi], 1u) == static_cast<unsigned>(n_tiles - 1);
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  if (i < n) {
+    const int rank = __ldcg(&rank_acc[i]);
+    keys_out[rank] = k;
+    idx_out[rank] = static_cast<uint32_t>(i);
+  }
+}
+
 __global__ void __launch_bounds__(kSmallThreads)
 small_hash_sort_kernel(const int32_t* __restrict__ tok_ids, const int64_t* __restrict__ tok_offsets,
                        const int64_t* __restrict__ ctx_key, int n, uint32_t weak, uint64_t* hash64, uint32_t* keys,
@@ -505,6 +562,27 @@ extern "C" int32_t ss_dedup_paths(const int32_t* tok_ids, const int64_t* tok_off
   const int warp_blocks = (n + warps_per_block - 1) / warps_per_block;
   SS_LAUNCH(hash_kernel, warp_blocks, warps_per_block * 32, 0, st, tok_ids, tok_offsets, ctx_key, n, weak, hash64,
             keys_a, idx_a);
+  if (n <= kRankSortMax) {                          // three launches: hash, sort by counting, match + rank + finalize
+    unsigned int* counters = reinterpret_cast<unsigned int*>(hist);      // the sort histogram is unused on this path
+    if (cudaMemsetAsync(counters, 0, 2 * sizeof(unsigned int), st) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return SS_ERR_CUDA;
+    }
+    // (idx_a holds the identity permutation the radix sort starts from: free here, it accumulates the ranks; the
+    //  group counters follow the two arrival counters in the histogram region)
+    const int n_groups = (n + kRankThreads - 1) / kRankThreads, n_tiles = (n + kRankTile - 1) / kRankTile;
+    if (cudaMemsetAsync(idx_a, 0, static_cast<size_t>(n) * sizeof(uint32_t), st) != cudaSuccess ||
+        cudaMemsetAsync(counters + 2, 0, static_cast<size_t>(n_groups) * sizeof(unsigned int), st) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return SS_ERR_CUDA;
+    }
+    SS_LAUNCH(rank_sort_kernel, n_groups * n_tiles, kRankThreads, 0, st, keys_a, n, n_tiles, reinterpret_cast<int*>(idx_a),
+              counters + 2, keys_b, idx_b);
+    SS_LAUNCH(small_match_finalize_kernel, (n + kSmallWarps - 1) / kSmallWarps, kSmallThreads, 0, st, keys_b, idx_b, n,
+              hash64, tok_ids, tok_offsets, ctx_key, slot_in, canon_out, rank, path_to_unique_out, unique_paths_out,
+              multiplicity_out, slot_out, num_unique_out, counters + 1);
+    return SS_OK;
+  }
   const int passes = weak ? 1 : 4;
   uint32_t *kin = keys_a, *kout = keys_b, *iin = idx_a, *iout = idx_b;
   for (int p = 0; p < passes; ++p) {

@@ -5,76 +5,25 @@
 // synchronisation, so that a caller that alternates between a few arenas and streams overlaps one step's copies
 // with another step's kernels.
 //
-// Rows nobody reads do not cross the bus: a duplicate candidate gets no forward pass (paper, Section "Computation
-// Deduplication"), so it has no query and no output of its own.  When the caller's q / out / lse buffers are
-// page-locked AND mapped (cudaHostAlloc / cudaHostRegister memory: the device can address them), the token ids go
-// first, the paths are deduplicated, and only then two small copy kernels move the query rows of the UNIQUE paths in
-// (read straight from the host buffer) and, after the attention, the live rows of out / lse back (written straight
-// into the host buffer) - how many rows those are is only known on the device, which is why kernels do it and not
-// cudaMemcpyAsync.  The copy kernels are a few persistent blocks, and the attention call is told to leave as many
-// SMs free (ss_attn_desc_t::max_sms): its tile and leaf blocks need an SM to themselves, and would otherwise wait
-// for a copy block that runs for as long as the bus takes.  Buffers that are not mapped take the plain path: every
-// logical candidate's rows are copied with cudaMemcpyAsync.
+// Rows nobody reads need not come back over the bus: a duplicate candidate gets no forward pass (paper, Section
+// "Computation Deduplication"), so it has no output of its own.  With SS_STEP_COMPACT_TRANSFERS, and out / lse
+// page-locked and mapped into the device's address space, only the live rows of out / lse - the first
+// u_q_offsets[num_unique], a number only the device knows - are returned, by a small kernel that writes them
+// straight into the host buffers.  The query rows still go in whole, with one cudaMemcpyAsync: fetching only the
+// unique paths' rows was measured and is not kept - as one copy per run of unique paths (after a host wait for the
+// deduplication) the ~2700 copies of a C5 step cost more than the 20 % of the bytes they save (each costs about as
+// much bus time as the 512 KB gap it skips, and the wait keeps the steps from overlapping: 135 ms per step against
+// 98 ms), and as a kernel reading mapped host memory the two directions together reach only 56-80 GB/s against the
+// 96 GB/s of two copy engines.
 #include "common.cuh"
 
 namespace ss {
 namespace host_step {
 
-constexpr int kCopyBlocks = 8;       // persistent blocks per copy kernel
+constexpr int kCopyBlocks = 8;       // persistent blocks of the copy kernel (8 reach 52 GB/s on the measured system)
 constexpr int kCopyThreads = 512;
-constexpr int kGatherBatch = 128;    // paths whose descriptors a block stages at a time
 
-// Query rows of the live unique paths, host -> device: path u's rows [u_q_src[u], + T) of the caller's buffer become
-// rows [u_q_offsets[u], + T) of the compact device buffer (a path's rows are contiguous on both sides; a batch of
-// consecutive paths is contiguous on the device side).  16-byte chunks, several in flight per thread.
-__global__ void __launch_bounds__(kCopyThreads)
-gather_q_from_host_kernel(const uint4* __restrict__ q_host, uint4* __restrict__ q_dev, const int32_t* __restrict__ num_unique,
-                          int32_t n_paths, const int64_t* __restrict__ u_q_offsets, const int64_t* __restrict__ u_q_src,
-                          int64_t row_chunks, int32_t* __restrict__ batch_counter) {
-  ss::grid_dependency_enter();
-  __shared__ int64_t s_off[kGatherBatch + 1], s_src[kGatherBatch];
-  __shared__ int s_batch;
-  int live = *num_unique;
-  live = live < 0 ? 0 : (live > n_paths ? n_paths : live);
-  for (;;) {
-    __syncthreads();
-    if (threadIdx.x == 0) s_batch = atomicAdd(batch_counter, 1);
-    __syncthreads();
-    const int p0 = s_batch * kGatherBatch;
-    if (p0 >= live) break;
-    const int np = min(kGatherBatch, live - p0);
-    for (int i = threadIdx.x; i <= np; i += blockDim.x) {
-      s_off[i] = u_q_offsets[p0 + i];
-      if (i < np) s_src[i] = u_q_src[p0 + i];
-    }
-    __syncthreads();
-    const int64_t row0 = s_off[0];
-    const int64_t n_chunks = (s_off[np] - row0) * row_chunks;
-    uint4* dst = q_dev + row0 * row_chunks;
-    for (int64_t c0 = threadIdx.x; c0 < n_chunks; c0 += 4LL * blockDim.x) {
-      uint4 v[4];
-#pragma unroll
-      for (int x = 0; x < 4; ++x) {
-        const int64_t c = c0 + static_cast<int64_t>(x) * blockDim.x;
-        if (c >= n_chunks) break;
-        const int64_t row = row0 + c / row_chunks;
-        int lo = 0, hi = np;                               // path of the batch that owns the row
-        while (hi - lo > 1) {
-          const int mid = (lo + hi) >> 1;
-          if (s_off[mid] <= row) lo = mid; else hi = mid;
-        }
-        v[x] = q_host[(s_src[lo] + (row - s_off[lo])) * row_chunks + c % row_chunks];
-      }
-#pragma unroll
-      for (int x = 0; x < 4; ++x) {
-        const int64_t c = c0 + static_cast<int64_t>(x) * blockDim.x;
-        if (c < n_chunks) dst[c] = v[x];
-      }
-    }
-  }
-}
-
-// The live rows of out / lse, device -> host: rows [0, u_q_offsets[U]) of the compact device buffers.
+// The live rows of out / lse, device -> (mapped) host: rows [0, u_q_offsets[U]) of the compact device buffers.
 __global__ void __launch_bounds__(kCopyThreads)
 rows_to_host_kernel(const uint4* __restrict__ out_dev, uint4* __restrict__ out_host, const uint4* __restrict__ lse_dev,
                     uint4* __restrict__ lse_host, const int32_t* __restrict__ num_unique, int32_t n_paths,
@@ -86,13 +35,13 @@ rows_to_host_kernel(const uint4* __restrict__ out_dev, uint4* __restrict__ out_h
   const int64_t tid = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   const int64_t nt = static_cast<int64_t>(gridDim.x) * blockDim.x;
   const int64_t n_out = rows * out_row_chunks;
-  for (int64_t c0 = tid; c0 < n_out; c0 += 4 * nt) {
-    uint4 v[4];
+  for (int64_t c0 = tid; c0 < n_out; c0 += 8 * nt) {
+    uint4 v[8];
 #pragma unroll
-    for (int x = 0; x < 4; ++x)
+    for (int x = 0; x < 8; ++x)
       if (c0 + x * nt < n_out) v[x] = out_dev[c0 + x * nt];
 #pragma unroll
-    for (int x = 0; x < 4; ++x)
+    for (int x = 0; x < 8; ++x)
       if (c0 + x * nt < n_out) out_host[c0 + x * nt] = v[x];
   }
   if (lse_host) {
@@ -114,7 +63,6 @@ struct Arena {                       // device-side layout of one step
   int32_t* num_unique;
   int32_t* u_leaf; int32_t* u_q_len; int64_t* u_q_offsets; int64_t* u_q_src;
   void* out; float* lse; int32_t* survivors; uint8_t* keep;
-  int32_t* copy_counter;             // batch counter of the query gather (zeroed every step)
   // workspaces of the three calls
   void* dedup_ws; size_t dedup_ws_bytes;
   void* attn_ws; size_t attn_ws_bytes;
@@ -125,9 +73,7 @@ struct Arena {                       // device-side layout of one step
 static size_t at_least_one(int64_t n) { return static_cast<size_t>(n > 0 ? n : 1); }
 
 // The attention descriptor of this step: the caller's resident fields + the staged per-path arrays.
-// `compact_q`: the device buffer holds the unique paths' rows at u_q_offsets (gathered from the host); otherwise it
-// holds every logical candidate's rows and the attention reads them in place through u_q_src.
-static ss_attn_desc_t step_desc(const ss_host_step_t& s, const Arena& a, bool compact_q = false, int max_sms = 0) {
+static ss_attn_desc_t step_desc(const ss_host_step_t& s, const Arena& a) {
   ss_attn_desc_t d = *s.attn;
   d.num_paths = s.n_paths;
   d.num_paths_dev = a.num_unique;
@@ -135,9 +81,8 @@ static ss_attn_desc_t step_desc(const ss_host_step_t& s, const Arena& a, bool co
   d.path_q_len = a.u_q_len;
   d.q_offsets = a.u_q_offsets;
   d.total_q = s.total_q;
-  d.q_src_offsets = compact_q ? nullptr : a.u_q_src;
-  d.q_src_rows = compact_q ? 0 : s.total_q;
-  d.max_sms = max_sms;
+  d.q_src_offsets = a.u_q_src;
+  d.q_src_rows = s.total_q;
   d.q = a.q;
   d.out = a.out;
   d.lse = a.lse;
@@ -172,7 +117,6 @@ static int32_t carve(const ss_host_step_t& s, void* base, Arena* a) {
   a->lse = c.take<float>(at_least_one(s.total_q) * static_cast<size_t>(s.attn->num_q_heads));
   a->survivors = c.take<int32_t>(P * static_cast<size_t>(s.top_k));
   a->keep = c.take<uint8_t>(N);
-  a->copy_counter = c.take<int32_t>(4);
   int32_t rc = ss_dedup_workspace_bytes(s.n_paths, &a->dedup_ws_bytes);
   if (rc != SS_OK) return rc;
   a->dedup_ws = c.take<char>(a->dedup_ws_bytes);
@@ -190,6 +134,7 @@ static int32_t carve(const ss_host_step_t& s, void* base, Arena* a) {
 static int32_t check(const ss_host_step_t* s) {
   if (!s || s->struct_size != sizeof(ss_host_step_t) || !s->attn) return SS_ERR_INVALID_ARG;
   if (s->attn->struct_size != sizeof(ss_attn_desc_t)) return SS_ERR_INVALID_ARG;
+  if (s->flags & ~SS_STEP_COMPACT_TRANSFERS) return SS_ERR_INVALID_ARG;
   if (s->n_paths < 0 || s->n_segments < 0 || s->top_k < 1 || s->total_tok < 0 || s->total_q < 0)
     return SS_ERR_INVALID_ARG;
   if (s->attn->num_q_heads < 1 || s->attn->head_dim < 1) return SS_ERR_INVALID_ARG;
@@ -243,7 +188,6 @@ extern "C" int32_t ss_candidate_step_host(const ss_host_step_t* step, void* devi
   const size_t N = static_cast<size_t>(s.n_paths), P = static_cast<size_t>(s.n_segments);
   const size_t row = static_cast<size_t>(s.attn->num_q_heads) * static_cast<size_t>(s.attn->head_dim);
   const size_t q_bytes = static_cast<size_t>(s.total_q) * row * sizeof(__nv_bfloat16);
-  const size_t lse_bytes = static_cast<size_t>(s.total_q) * static_cast<size_t>(s.attn->num_q_heads) * sizeof(float);
 
   // ---- host -> device: the step's candidates, queries and scores ------------------------------------------------
   const cudaMemcpyKind H2D = cudaMemcpyHostToDevice, D2H = cudaMemcpyDeviceToHost;
@@ -254,28 +198,15 @@ extern "C" int32_t ss_candidate_step_host(const ss_host_step_t* step, void* devi
   SS_COPY(a.path_leaf_node, s.path_leaf_node, N * 4, H2D);
   SS_COPY(a.path_q_len, s.path_q_len, N * 4, H2D);
   SS_COPY(a.q_offsets, s.q_offsets, (N + 1) * 8, H2D);
-  // mapped q / out / lse: only the unique paths' rows cross the bus (see the top of the file)
-  void *q_map = nullptr, *out_map = nullptr, *lse_map = nullptr;
-  bool slim = s.total_q > 0 && s.n_paths > 0 && row * sizeof(__nv_bfloat16) % 16 == 0;
-  if (slim && (cudaHostGetDevicePointer(&q_map, const_cast<void*>(s.q), 0) != cudaSuccess ||
-               cudaHostGetDevicePointer(&out_map, s.out, 0) != cudaSuccess ||
-               (s.lse && cudaHostGetDevicePointer(&lse_map, s.lse, 0) != cudaSuccess))) {
+  SS_COPY(a.q, s.q, q_bytes, H2D);
+  // compact return: needs out / lse mapped (the kernel writes them) and whole 16-byte chunks per row
+  void *out_map = nullptr, *lse_map = nullptr;
+  bool compact = (s.flags & SS_STEP_COMPACT_TRANSFERS) != 0 && s.total_q > 0 && s.n_paths > 0 &&
+                 row * sizeof(__nv_bfloat16) % 16 == 0;
+  if (compact && (cudaHostGetDevicePointer(&out_map, s.out, 0) != cudaSuccess ||
+                  (s.lse && cudaHostGetDevicePointer(&lse_map, s.lse, 0) != cudaSuccess))) {
     (void)cudaGetLastError();
-    slim = false;
-  }
-  int dev_sms = 0;
-  if (slim) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&dev_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
-        dev_sms <= 4 * kCopyBlocks) {
-      (void)cudaGetLastError();
-      slim = false;
-    }
-  }
-  if (slim) {
-    if (cudaMemsetAsync(a.copy_counter, 0, 16, st) != cudaSuccess) { (void)cudaGetLastError(); return SS_ERR_CUDA; }
-  } else {
-    SS_COPY(a.q, s.q, q_bytes, H2D);
+    compact = false;
   }
   SS_COPY(a.scores, s.scores, N * 4, H2D);
   SS_COPY(a.seg_offsets, s.seg_offsets, (P + 1) * 4, H2D);
@@ -288,13 +219,17 @@ extern "C" int32_t ss_candidate_step_host(const ss_host_step_t* step, void* devi
   rc = ss_gather_unique_paths(a.unique_paths, a.num_unique, s.n_paths, a.path_leaf_node, a.path_q_len, a.q_offsets,
                               a.u_leaf, a.u_q_len, a.u_q_offsets, a.u_q_src, stream);
   if (rc != SS_OK) return rc;
-  const int64_t row_chunks = static_cast<int64_t>(row * sizeof(__nv_bfloat16) / 16);
-  if (slim)
-    SS_LAUNCH(gather_q_from_host_kernel, kCopyBlocks, kCopyThreads, 0, st, static_cast<const uint4*>(q_map),
-              static_cast<uint4*>(a.q), static_cast<const int32_t*>(a.num_unique), s.n_paths,
-              static_cast<const int64_t*>(a.u_q_offsets), static_cast<const int64_t*>(a.u_q_src), row_chunks, a.copy_counter);
-  // (two copy kernels of other steps may be running beside this step's attention: their SMs are left alone)
-  const ss_attn_desc_t d = step_desc(s, a, slim, slim ? dev_sms - 2 * kCopyBlocks : 0);
+  ss_attn_desc_t d = step_desc(s, a);
+  if (compact && d.max_sms == 0) {
+    // the copy kernel of the step before this one (another stream) runs for as long as the bus takes and needs SMs
+    // that this step's persistent attention blocks do not hold
+    int dev = 0, n_sm = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess &&
+        n_sm > 4 * kCopyBlocks)
+      d.max_sms = n_sm - 2 * kCopyBlocks;
+    else
+      (void)cudaGetLastError();
+  }
   rc = ss_tree_attention(&d, a.attn_ws, a.attn_ws_bytes, stream);
   if (rc != SS_OK) return rc;
   rc = ss_topk_prune(a.scores, a.seg_offsets, s.n_segments, s.n_paths, s.top_k, a.survivors, a.keep, a.topk_ws,
@@ -309,14 +244,14 @@ extern "C" int32_t ss_candidate_step_host(const ss_host_step_t* step, void* devi
   if (s.slot_out) SS_COPY(s.slot_out, a.slot_out, N * 4, D2H);
   SS_COPY(s.num_unique, a.num_unique, 4, D2H);
   SS_COPY(s.u_q_offsets, a.u_q_offsets, (N + 1) * 8, D2H);
-  if (slim) {
+  if (compact) {
     SS_LAUNCH(rows_to_host_kernel, kCopyBlocks, kCopyThreads, 0, st, static_cast<const uint4*>(a.out),
               static_cast<uint4*>(out_map), reinterpret_cast<const uint4*>(a.lse), static_cast<uint4*>(lse_map),
-              static_cast<const int32_t*>(a.num_unique), s.n_paths, static_cast<const int64_t*>(a.u_q_offsets), row_chunks,
-              static_cast<int64_t>(s.attn->num_q_heads) * 4);
+              static_cast<const int32_t*>(a.num_unique), s.n_paths, static_cast<const int64_t*>(a.u_q_offsets),
+              static_cast<int64_t>(row * sizeof(__nv_bfloat16) / 16), static_cast<int64_t>(s.attn->num_q_heads) * 4);
   } else {
     SS_COPY(s.out, a.out, q_bytes, D2H);
-    if (s.lse) SS_COPY(s.lse, a.lse, lse_bytes, D2H);
+    if (s.lse) SS_COPY(s.lse, a.lse, static_cast<size_t>(s.total_q) * static_cast<size_t>(s.attn->num_q_heads) * sizeof(float), D2H);
   }
   SS_COPY(s.survivors, a.survivors, P * static_cast<size_t>(s.top_k) * 4, D2H);
   SS_COPY(s.keep, a.keep, N, D2H);

@@ -41,13 +41,18 @@ __device__ void bitonic_sort(uint64_t* keys, int n_pad) {
 }
 
 __global__ void __launch_bounds__(kThreads)
-topk_kernel(const float* __restrict__ scores, const int32_t* __restrict__ seg_offsets, int k,
-            int32_t* __restrict__ survivors, uint8_t* __restrict__ keep, uint64_t* __restrict__ scratch) {
+topk_kernel(const float* __restrict__ scores, const int32_t* __restrict__ seg_offsets, int n_total, int k,
+            int32_t* __restrict__ survivors, uint8_t* __restrict__ keep, uint64_t* __restrict__ scratch,
+            int32_t* __restrict__ status) {
   ss::grid_dependency_enter();
   __shared__ uint64_t smem_keys[kSmemKeys];
   const int s = blockIdx.x;
   const int lo = seg_offsets[s], hi = seg_offsets[s + 1];
-  const int n = hi - lo;
+  // a segment that does not lie inside [0, n_total] is reported and treated as empty: its offsets index keep[] and
+  // the scratch region, so following them would write out of bounds
+  const bool bad = lo < 0 || hi < lo || hi > n_total;
+  if (bad && threadIdx.x == 0) set_status(status, SS_ERR_BAD_INPUT);
+  const int n = bad ? 0 : hi - lo;
   if (n <= 0) {
     for (int j = threadIdx.x; j < k; j += blockDim.x) survivors[static_cast<int64_t>(s) * k + j] = -1;
     return;
@@ -76,14 +81,17 @@ topk_kernel(const float* __restrict__ scores, const int32_t* __restrict__ seg_of
 //   all verified -> final, selected = the k best.
 __global__ void __launch_bounds__(kThreads)
 early_prune_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ verified,
-                   const int32_t* __restrict__ seg_offsets, int k, uint8_t* __restrict__ pruned,
-                   int32_t* __restrict__ selected, uint8_t* __restrict__ final_out, uint64_t* __restrict__ scratch) {
+                   const int32_t* __restrict__ seg_offsets, int n_total, int k, uint8_t* __restrict__ pruned,
+                   int32_t* __restrict__ selected, uint8_t* __restrict__ final_out, uint64_t* __restrict__ scratch,
+                   int32_t* __restrict__ status) {
   ss::grid_dependency_enter();
   __shared__ uint64_t smem_keys[kSmemKeys];
   __shared__ int s_nver, s_nperfect;
   const int s = blockIdx.x;
   const int lo = seg_offsets[s], hi = seg_offsets[s + 1];
-  const int n = hi - lo;
+  const bool bad = lo < 0 || hi < lo || hi > n_total;        // (see topk_kernel)
+  if (bad && threadIdx.x == 0) set_status(status, SS_ERR_BAD_INPUT);
+  const int n = bad ? 0 : hi - lo;
   for (int j = threadIdx.x; j < k; j += blockDim.x) selected[static_cast<int64_t>(s) * k + j] = -1;
   if (n <= 0) {
     if (threadIdx.x == 0) final_out[s] = 1;      // nothing left to verify in an empty segment
@@ -159,14 +167,17 @@ extern "C" int32_t ss_early_prune(const float* scores, const uint8_t* verified, 
   size_t need = 0;
   ss_topk_workspace_bytes(n_total, &need);
   if (workspace_bytes < need) return SS_ERR_WORKSPACE_TOO_SMALL;
-  SS_LAUNCH(topk::early_prune_kernel, n_segments, topk::kThreads, 0, st, scores, verified, seg_offsets, k, pruned_out,
-            selected_out, final_out, static_cast<uint64_t*>(workspace));
+  if (cudaMemsetAsync(workspace, 0, sizeof(int32_t), st) != cudaSuccess) { (void)cudaGetLastError(); return SS_ERR_CUDA; }
+  SS_LAUNCH(topk::early_prune_kernel, n_segments, topk::kThreads, 0, st, scores, verified, seg_offsets, n_total, k,
+            pruned_out, selected_out, final_out, reinterpret_cast<uint64_t*>(static_cast<char*>(workspace) + kAlign),
+            static_cast<int32_t*>(workspace));
   return SS_OK;
 }
 
 extern "C" int32_t ss_topk_workspace_bytes(int32_t n_total, size_t* out_bytes) {
   if (n_total < 0 || !out_bytes) return SS_ERR_INVALID_ARG;
-  *out_bytes = ss::align_up(static_cast<size_t>(2) * (n_total > 0 ? n_total : 1) * sizeof(uint64_t));
+  // the status word (first bytes, see ss_last_device_status), then two 64-bit sort keys per candidate
+  *out_bytes = ss::kAlign + ss::align_up(static_cast<size_t>(2) * (n_total > 0 ? n_total : 1) * sizeof(uint64_t));
   return SS_OK;
 }
 
@@ -194,7 +205,8 @@ extern "C" int32_t ss_topk_prune(const float* scores, const int32_t* seg_offsets
     (void)cudaGetLastError();
     return SS_ERR_CUDA;
   }
-  SS_LAUNCH(topk::topk_kernel, n_segments, topk::kThreads, 0, st, scores, seg_offsets, k, survivors_out, keep_out,
-            static_cast<uint64_t*>(workspace));
+  if (cudaMemsetAsync(workspace, 0, sizeof(int32_t), st) != cudaSuccess) { (void)cudaGetLastError(); return SS_ERR_CUDA; }
+  SS_LAUNCH(topk::topk_kernel, n_segments, topk::kThreads, 0, st, scores, seg_offsets, n_total, k, survivors_out, keep_out,
+            reinterpret_cast<uint64_t*>(static_cast<char*>(workspace) + kAlign), static_cast<int32_t*>(workspace));
   return SS_OK;
 }

@@ -142,8 +142,9 @@ class HostStepPipeline:
     the device).  submit(i) enqueues one whole step on set i and returns at once; alternating the sets overlaps the
     copies of one step with the kernels of another."""
 
-    def __init__(self, resident: DevicePipeline, depth: int = 2):
+    def __init__(self, resident: DevicePipeline, depth: int = 2, compact: bool = False):
         self.resident = resident
+        self.compact = compact
         w, dev = resident.w, resident.device
         self.device = dev
         N, P, k = w.num_paths, resident.P, w.top_k
@@ -176,16 +177,17 @@ class HostStepPipeline:
                 keep=pin((max(N, 1),), torch.uint8), device_status=pin((1,), torch.int32))
             step = B.make_host_step(resident.desc, n_paths=N, n_segments=P, top_k=k,
                                     total_tok=int(w.tok_offsets[-1]), total_q=tq, host_in=h_in, host_out=h_out,
-                                    dedup_flags=resident.dedup_flags)
+                                    dedup_flags=resident.dedup_flags,
+                                    flags=B.SS_STEP_COMPACT_TRANSFERS if compact else 0)
             arena = B.alloc_workspace(B.ss_candidate_step_host_arena_bytes(step), dev)
             self.sets.append(dict(h_in=h_in, h_out=h_out, step=step, arena=arena, stream=torch.cuda.Stream(dev)))
         self.h2d_bytes = sum(t.numel() * t.element_size() for t in self.sets[0]["h_in"].values())
         self.d2h_bytes = sum(t.numel() * t.element_size() for t in self.sets[0]["h_out"].values())
 
     def measure_traffic(self):
-        """Runs one step on set 0 and sets h2d_bytes / d2h_bytes to what that step moved over the bus.  Page-locked
-        buffers from torch are mapped, so the call fetches only the unique paths' query rows and returns only the live
-        rows of out / lse; whether it did is read off a sentinel row past the live ones (left untouched if so)."""
+        """Runs one step on set 0 and sets d2h_bytes to what that step moved back over the bus.  With
+        SS_STEP_COMPACT_TRANSFERS (and page-locked, hence mapped, buffers) only the live rows of out / lse come back;
+        that it happened is read off a sentinel row past the live ones (left untouched if so)."""
         s = self.sets[0]
         o, i = s["h_out"], s["h_in"]
         tq_all = o["out"].shape[0]
@@ -194,14 +196,12 @@ class HostStepPipeline:
         s["stream"].synchronize()
         U = int(o["num_unique"][0])
         tq_live = int(o["u_q_offsets"][U]) if self.resident.N else 0
-        slim = tq_live < tq_all and bool((o["out"][tq_all - 1].float() == -7.0).all())
-        if slim:
+        compact = tq_live < tq_all and bool((o["out"][tq_all - 1].float() == -7.0).all())
+        if compact:
             row = o["out"].shape[1] * o["out"].shape[2] * 2
-            small_in = sum(t.numel() * t.element_size() for k, t in i.items() if k != "q")
             small_out = sum(t.numel() * t.element_size() for k, t in o.items() if k not in ("out", "lse"))
-            self.h2d_bytes = small_in + tq_live * row
             self.d2h_bytes = small_out + tq_live * (row + o["lse"].shape[1] * 4)
-        return slim
+        return compact
 
     def submit(self, i: int):
         s = self.sets[i % len(self.sets)]

@@ -72,3 +72,33 @@ def test_all_verified_agrees_with_topk_prune():
     pruned, sel, fin = run(sc, np.ones(164, np.uint8), seg, 8)
     surv, keep = oracle.topk(sc, seg, 8)
     assert fin.all() and np.array_equal(sel, surv) and np.array_equal(1 - pruned, keep)
+
+
+def test_topk_and_early_prune_report_segments_outside_the_candidates():
+    """Segment offsets index keep[] / pruned[] and the scratch region: a segment that does not lie inside [0, n_total]
+    is reported through the status word and treated as empty, never followed."""
+    dev = torch.device(DEV)
+    n, k = 40, 3
+    scores = torch.rand(n, device=dev)
+    seg = torch.tensor([0, 10, 25, 4000], dtype=torch.int32, device=dev)      # the last segment runs past n
+    surv = torch.full((3, k), -9, dtype=torch.int32, device=dev)
+    keep = torch.full((n,), 7, dtype=torch.uint8, device=dev)
+    ws = B.alloc_workspace(B.ss_topk_workspace_bytes(n), dev)
+    B.ss_topk_prune(scores, seg, 3, n, k, surv, keep, ws)
+    torch.cuda.synchronize()
+    assert B.ss_last_device_status(ws) == B.SS_ERR_BAD_INPUT
+    assert surv[2].tolist() == [-1] * k and keep[25:].sum().item() == 0      # the bad segment selected nothing
+    s_ref, k_ref = oracle.topk(scores.cpu().numpy(), np.asarray([0, 10, 25], np.int32), k)
+    assert np.array_equal(surv[:2].cpu().numpy(), s_ref) and np.array_equal(keep[:25].cpu().numpy(), k_ref[:25])
+    ver = torch.ones(n, dtype=torch.uint8, device=dev)
+    pruned = torch.empty(n, dtype=torch.uint8, device=dev)
+    sel = torch.empty((3, k), dtype=torch.int32, device=dev)
+    fin = torch.empty(3, dtype=torch.uint8, device=dev)
+    seg_bad = torch.tensor([0, 10, 5, 40], dtype=torch.int32, device=dev)     # not monotone
+    B.ss_early_prune(scores, ver, seg_bad, 3, n, k, pruned, sel, fin, ws)
+    torch.cuda.synchronize()
+    assert B.ss_last_device_status(ws) == B.SS_ERR_BAD_INPUT
+    # a clean call clears the word again
+    B.ss_topk_prune(scores, torch.tensor([0, 10, 25, 40], dtype=torch.int32, device=dev), 3, n, k, surv, keep, ws)
+    torch.cuda.synchronize()
+    assert B.ss_last_device_status(ws) == B.SS_OK

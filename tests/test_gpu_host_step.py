@@ -66,21 +66,27 @@ def test_host_step_empty_batch_and_errors():
 
 
 @pytest.mark.parametrize("cfg", [2, 4])
-def test_host_step_moves_only_unique_rows_when_the_buffers_are_mapped(cfg):
-    """Page-locked buffers are mapped into the device's address space: the call then fetches the query rows of the unique
-    paths only and returns only the live rows of out / lse (a duplicate gets no forward pass, hence no query and no
-    output of its own).  Rows past the live ones must stay as the caller left them."""
+def test_host_step_with_compact_transfers_returns_only_live_rows(cfg):
+    """SS_STEP_COMPACT_TRANSFERS: only the live rows of out / lse come back (a duplicate gets no forward pass, hence no
+    output of its own).  Rows past the live ones must stay as the caller left them, and the results equal those of the
+    device-resident calls bit for bit."""
     w = synth.make_config(cfg)
     pipe = DevicePipeline(w, DEV)
     pipe.step()
     r_dev = pipe.results()
-    host = HostStepPipeline(pipe, depth=1)
+    host = HostStepPipeline(pipe, depth=2, compact=True)
     full_in, full_out = host.h2d_bytes, host.d2h_bytes
     assert host.measure_traffic()
     U, tq = r_dev["num_unique"], r_dev["total_q"]
     assert U < w.num_paths and tq < w.total_q
     row = w.num_q_heads * w.head_dim * 2
-    assert host.h2d_bytes == full_in - (w.total_q - tq) * row
+    assert host.h2d_bytes == full_in
     assert host.d2h_bytes == full_out - (w.total_q - tq) * (row + w.num_q_heads * 4)
-    r = host.results(0)
-    assert np.array_equal(r["out"], r_dev["out"]) and np.array_equal(r["lse"], r_dev["lse"])
+    for i in range(4):
+        host.submit(i)
+    host.synchronize()
+    for i in range(2):
+        r = host.results(i)
+        assert np.array_equal(r["out"], r_dev["out"]) and np.array_equal(r["lse"], r_dev["lse"])
+        for key in ("canon", "path_to_unique", "unique_paths", "multiplicity", "slot_out", "survivors", "keep"):
+            assert np.array_equal(r[key], r_dev[key]), key

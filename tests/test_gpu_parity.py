@@ -182,7 +182,8 @@ def dedup_case(rng, n, alphabet, max_len, n_ctx):
 
 @pytest.mark.parametrize("flags", [0, B.SS_FLAG_WEAK_HASH])
 @pytest.mark.parametrize("n,alphabet,max_len,n_ctx", [
-    (1, 3, 4, 1), (2, 2, 2, 1), (37, 2, 3, 2), (300, 3, 5, 2), (2049, 4, 6, 3), (4096, 3, 5, 2), (4097, 3, 5, 2), (5000, 2, 40, 1), (20000, 50, 3, 4),
+    (1, 3, 4, 1), (2, 2, 2, 1), (37, 2, 3, 2), (300, 3, 5, 2), (1025, 3, 5, 2), (2049, 4, 6, 3), (4096, 3, 5, 2), (4097, 3, 5, 2), (5000, 2, 40, 1), (8192, 3, 6, 2), (12000, 4, 6, 3),
+    (16384, 3, 5, 2), (16385, 3, 5, 2), (20000, 50, 3, 4),
 ])
 def test_dedup_random_collision_heavy(n, alphabet, max_len, n_ctx, flags):
     rng = np.random.default_rng(n * 31 + alphabet)
@@ -403,6 +404,41 @@ def test_attention_page_permutation_and_explicit_scale():
     r2, _ = attention_only(w, sm_scale=0.05)
     # only the physical page ids differ: every item sees the same numbers in the same order
     assert np.array_equal(r2["out"], r1["out"]) and np.array_equal(r2["lse"], r1["lse"])
+
+
+def test_attention_flat_per_path_page_tables():
+    """A cache that keeps one flat page list per sequence is the tree form with one node per path: a root that is its
+    own leaf, whose page list is the whole sequence.  Same pool, same queries: the results must agree with the oracle
+    on the flat description and (within the gates) with the shared-prefix description of the same data."""
+    import copy
+    w = synth.build_tree_workload("flat", 21, 8, 2, [64], [5], 2, (3, 150), lambda i, n, rng: 1 + (i % 2) * 23)
+    r_tree, ref = attention_only(w)
+    flat = copy.copy(w)
+    parents, lens, pages, offs = [], [], [], [0]
+    for p in range(w.num_paths):
+        chain, n = [], int(w.path_leaf_node[p])
+        while n >= 0:
+            chain.append(n)
+            n = int(w.node_parent[n])
+        pl, total = [], 0
+        for n in reversed(chain):                              # inner nodes hold whole pages, so the lists concatenate
+            pl += list(w.node_pages[w.node_page_offsets[n]:w.node_page_offsets[n + 1]])
+            total += int(w.node_kv_len[n])
+        parents.append(-1)
+        lens.append(total)
+        pages += pl
+        offs.append(len(pages))
+    flat.node_parent = np.asarray(parents, np.int32)
+    flat.node_kv_len = np.asarray(lens, np.int32)
+    flat.node_pages = np.asarray(pages, np.int32)
+    flat.node_page_offsets = np.asarray(offs, np.int64)
+    flat.path_leaf_node = np.arange(w.num_paths, dtype=np.int32)
+    flat.slot_in = flat.path_leaf_node.copy()
+    r_flat, ref_flat = attention_only(flat)
+    assert np.array_equal(ref_flat["unique_paths"], ref["unique_paths"])
+    o_ref, l_ref = oracle.tree_attention_workload(flat, paths=ref_flat["unique_paths"])
+    tight_gates(r_flat["out"], o_ref, np.abs(r_flat["lse"] - l_ref).max(), 0)
+    assert np.abs(r_flat["out"] - r_tree["out"]).max() <= 2 * TIGHT_ABS + TIGHT_REL * np.abs(o_ref).max()
 
 
 def test_attention_empty_and_degenerate():

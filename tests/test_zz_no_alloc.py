@@ -55,9 +55,10 @@ def test_static_scratch_dedup_matches_workspace_dedup_twice_in_a_row():
 
 
 def test_static_scratch_dedup_small_and_empty_batches():
-    # batches of at most 4096 paths take the two-launch path, whose arrival counters live inside the shared scratch and
+    # batches of at most 4096 paths take the two-launch path and batches of up to 32768 the three-launch one: their
+    # arrival counters live inside the shared scratch and
     # must start at zero on every call; n = 0 writes only the count
-    for seed, n in [(3, 4096), (4, 300), (5, 1), (6, 4096)]:
+    for seed, n in [(3, 4096), (4, 300), (5, 1), (6, 4096), (8, 16384), (9, 16385)]:
         ids, off, ctx, slot = _case(seed, n)
         want = _run(False, ids, off, ctx, slot, n)
         got = _run(True, ids, off, ctx, slot, n)
