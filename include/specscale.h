@@ -14,6 +14,9 @@
  *   - All work is enqueued on the caller's CUDA stream, passed as void* (a cudaStream_t; NULL = the legacy
  *     default stream).  No entry point synchronises the host with the device, except
  *     ss_last_device_status, which exists to do exactly that.
+ *   - Host threads: calls may come from several host threads as long as calls that share a workspace, an arena or a
+ *     stream do not overlap; the once-per-device set-up some calls do on first use (kernel attributes, the static
+ *     scratch address) is idempotent.  The ss_profile_* diagnostics are for a single-threaded harness.
  *   - Every function returns an int32_t status.  Argument errors are detected on the host before any launch.
  *     Errors that only the device can see (an unsupported tree shape, a workspace that turns out too small
  *     for the tree, a bounded wait that expired) are recorded in the first bytes of the workspace and read

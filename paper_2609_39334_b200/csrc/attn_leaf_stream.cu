@@ -87,7 +87,10 @@ template <int NT, int WARPS, int STAGES>
 __global__ void __launch_bounds__(WARPS * 32, 1)
 leaf_stream_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
                    const __grid_constant__ Params P) {
-  ss::grid_dependency_enter();
+  // This kernel follows the tile kernel but its items need nothing from it: it starts as soon as SMs are free (the
+  // tile kernel has waited for the planner before releasing it) and waits for the tile kernel only where it first
+  // reads the shared-node partials - and in every thread before the kernel ends.
+  ss::grid_dependency_release();
   using C = Cfg<NT, WARPS, STAGES>;
   constexpr int kStages = STAGES;
   SS_STAMP_BEGIN(P.hdr, 4);
@@ -111,8 +114,10 @@ leaf_stream_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
   fence_barrier_init();
   __syncthreads();
 
-  const bool plan_ok = P.hdr->status == SS_OK;
-  const int n_items = plan_ok ? P.hdr->n_leaf_items : 0;
+  // (what the planner wrote is read from L2 until the dependency wait: this kernel's blocks start while the tile
+  //  kernel is still running, on SMs whose L1 may hold lines from before the planner ran)
+  const bool plan_ok = __ldcg(&P.hdr->status) == SS_OK;
+  const int n_items = plan_ok ? __ldcg(&P.hdr->n_leaf_items) : 0;
   const int G = P.G;
   const float c = P.scale_log2;
   const float lazy_raw = kLazyLog2 / c;
@@ -127,7 +132,12 @@ leaf_stream_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     f_e = __shfl_sync(0xffffffffu, e, 0);
   };
   auto fetch_desc = [&]() {                                      // step 2: its descriptor
-    if (f_e < n_items) f_it = P.leaf_items[f_e];
+    if (f_e < n_items) {
+      const uint4* src = reinterpret_cast<const uint4*>(P.leaf_items + f_e);
+      const uint4 lo = __ldcg(src), hi = __ldcg(src + 1);
+      *reinterpret_cast<uint4*>(&f_it) = lo;
+      *(reinterpret_cast<uint4*>(&f_it) + 1) = hi;
+    }
   };
   auto fetch_finish = [&](Item& it) {                            // step 3: page ids, query rows
     it.valid = f_e < n_items ? 1 : 0;
@@ -139,7 +149,7 @@ leaf_stream_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                     f_it.q_src < (P.q_src_offsets ? P.q_src_rows : P.total_q),
                 &P.hdr->status, { it.valid = 0; return; });
     it.my_page = lane < it.n_pages ? P.node_pages[static_cast<int64_t>(f_it.page0) + lane] : 0;
-    it.chunks = P.dec_leaf_chunks[f_it.dec];
+    it.chunks = __ldcg(&P.dec_leaf_chunks[f_it.dec]);
     // B fragments of Q^T: thread (gid, tig) holds Q[row 8 nt + gid][dims 16 ks + 2 tig, + 1] and the same 8 dims on
     const uint32_t* q0 = reinterpret_cast<const uint32_t*>(P.q + (static_cast<int64_t>(f_it.q_src) * P.Hq + it.g * G) * kHeadDim);
 #pragma unroll
@@ -306,6 +316,7 @@ leaf_stream_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       issue_one();
     }
     if (!ok) break;
+    ss::grid_dependency_wait();       // the tile kernel's partials are complete from here on (returns at once later)
 
     // ---- the item's normalised partial ---------------------------------------------------------------------------------
 #pragma unroll
@@ -425,8 +436,10 @@ leaf_stream_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       ++n_cons;
     }
     if (lane == 0) set_status(&P.hdr->status, SS_ERR_TIMEOUT);
+    ss::grid_dependency_wait();
     return;
   }
+  ss::grid_dependency_wait();         // (every thread, before the sweeps below and before the kernel ends)
   if (!plan_ok) return;
 
   // ---- decode tokens without a private leaf (empty or shared): their partials all come from the tile kernel -------------

@@ -76,7 +76,7 @@ __device__ __forceinline__ ItemView view(const TileItem& it) {
 __global__ void __launch_bounds__(kUmmaThreads, 2)
 tile_items_umma_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
                        const Params P) {
-  ss::grid_dependency_enter();
+  ss::grid_dependency_enter_then_release();   // (the leaf kernel behind this one starts without waiting for it)
   extern __shared__ __align__(1024) uint8_t smem[];
   Ctrl& C = *reinterpret_cast<Ctrl*>(smem + kOffCtrl);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;

@@ -48,6 +48,10 @@ constexpr int kStageBytes = kTile * 256;       // one K or V tile: [16 groups of
 constexpr int kStagesK = 3;
 constexpr int kStagesV = 2;                    // V is consumed a softmax later than K: two stages are enough
 constexpr int kRing = 3;                       // S/P buffers
+#ifndef SS_PRE_ISSUE
+#define SS_PRE_ISSUE 2
+#endif
+constexpr int kPreIssue = SS_PRE_ISSUE;        // Q K^T products of the next item issued before the current one ends (< kRing)
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColS = 0;                  // kRing x kTile columns
 constexpr uint32_t kColO = kRing * kTile;      // 128 columns
@@ -142,7 +146,7 @@ __device__ __noinline__ void exact_second_pass(const Params& P, const TileItem* 
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
                             const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ Params P) {
-  ss::grid_dependency_enter();
+  ss::grid_dependency_enter_then_release();   // (the leaf kernel behind this one starts without waiting for it)
   extern __shared__ __align__(1024) uint8_t smem[];
   __shared__ Ctrl C;
   SS_STAMP_BEGIN(P.hdr, 2);
@@ -233,7 +237,8 @@ tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const _
 
   if (tid == 0) fetch_item(0);
   __syncthreads();
-  bool q_pending = false;   // V producer warp: a gather of the coming item's Q rows is under way
+  bool q_pending = false;   // V producer warp: the gather of the first item's Q rows is under way
+  int qk_pre = 0;           // Q K^T issuer warp: products of the coming item that were issued during the one before
   if (warp == kSoftmaxWarps + 1) {                               // Q of a first stacked item
     if (__all_sync(0xffffffffu, mbar_wait(&C.item_ready[0], 0, abort_flag))) {
       const int e0 = C.item_e[0];
@@ -252,8 +257,15 @@ tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const _
     }
   }
 
+#ifdef SS_STAMPS
+  long long tl_wait = 0, tl_ld = 0, tl_ref = 0, tl_exp = 0, tl_store = 0, tl_mark = 0, tl_tiles = 0;
+  long long acc_first_s = 0, acc_tiles = 0, acc_o_wait = 0, acc_epi = 0, acc_sync = 0, acc_items = 0, t_mark = 0;
+#endif
   for (;;) {
     const int slot = item_seq & 1;
+#ifdef SS_STAMPS
+    if (tid == 0) t_mark = clock64();
+#endif
     // the descriptor of this item was published during the previous one (or before the loop)
     bool have = mbar_wait(&C.item_ready[slot], (item_seq >> 1) & 1, abort_flag);
     const int e = have ? C.item_e[slot] : -1;
@@ -300,11 +312,23 @@ tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const _
         for (int j = 0; j < n_tiles; ++j) {
           const uint32_t gj = g_tile + j;
           const uint32_t s_col = kColS + b * kTile + hf * 64;     // this thread's 64 scores; its P goes over the first 32
+#ifdef SS_STAMPS
+          if (tid == 0) tl_mark = clock64();
+#endif
           if (!mbar_wait(&C.s_full[b], b_phase, abort_flag)) ok = false;
+#ifdef SS_STAMPS
+          if (tid == 0 && j > 0) { const long long t = clock64(); tl_wait += t - tl_mark; tl_mark = t; }
+#endif
+#ifdef SS_STAMPS
+          if (tid == 0 && j == 0) { const long long t = clock64(); acc_first_s += t - t_mark; t_mark = t; }
+#endif
           tc_fence_after();
           uint32_t sr[64];
           tmem_ld32(tmem + lane_base + s_col, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
           tmem_wait_ld();
+#ifdef SS_STAMPS
+          if (tid == 0 && j > 0) { const long long t = clock64(); tl_ld += t - tl_mark; tl_mark = t; }
+#endif
           tmem_ld32(tmem + lane_base + s_col + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
 
           const bool masked = j >= first_masked_tile;             // warp-uniform
@@ -352,6 +376,9 @@ tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const _
               l *= alpha;
             }
           }
+#ifdef SS_STAMPS
+          if (tid == 0 && j > 0) { const long long t = clock64(); tl_ref += t - tl_mark; tl_mark = t; }
+#endif
           const float mc = m * cl2;
           const f32x2 cl2_2 = pack2(cl2, cl2);
           const f32x2 nmc2 = pack2(-mc, -mc);
@@ -375,6 +402,9 @@ tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const _
               if ((c & 14) == 0) mx4[(c >> 4) & 3] = max3(mx4[(c >> 4) & 3], s0, s1);   // every eighth pair
             }
           }
+#ifdef SS_STAMPS
+          if (tid == 0 && j > 0) { const long long t = clock64(); tl_exp += t - tl_mark; tl_mark = t; }
+#endif
           float sum4[4];
           unpack2(sum2[0], sum4[0], sum4[1]);
           unpack2(sum2[1], sum4[2], sum4[3]);
@@ -420,18 +450,27 @@ tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const _
           tmem_wait_st();
           tc_fence_before();
           mbar_arrive(&C.p_full[b]);
+#ifdef SS_STAMPS
+          if (tid == 0 && j > 0) { const long long t = clock64(); tl_store += t - tl_mark; ++tl_tiles; }
+#endif
           if (++b == kRing) { b = 0; b_phase ^= 1u; }
           tag_prev = tag;
           if (par) tag ^= 3u;                                     // (the tag changes with every second tile: 1 <-> 2)
           par ^= 1u;
         }
         ok = __all_sync(0xffffffffu, ok);
+#ifdef SS_STAMPS
+        if (tid == 0) { const long long t = clock64(); acc_tiles += t - t_mark; t_mark = t; }
+#endif
         if (ok) {
           ok = mbar_wait(&C.o_final, q_uses & 1, abort_flag);
           ok = __all_sync(0xffffffffu, ok);
           tc_fence_after();
         }
       }
+#ifdef SS_STAMPS
+      if (tid == 0) { const long long t = clock64(); acc_o_wait += t - t_mark; t_mark = t; }
+#endif
       // ---- epilogue: the two halves add their row sums; each writes 64 output columns ---------------------------------
       C.xmax[0][hf][row] = __float_as_uint(l);                  // (every tile of the item is behind both halves here)
       pair_barrier();
@@ -610,26 +649,35 @@ tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const _
           // Q buffer slot ^ 1 is free: the products of the item before this one have completed
           if (which == 0 && nv.n_tiles > 0 && nv.kind == kItemChain && elect_one()) q_tma_start(nv, slot ^ 1);
           // Q buffer slot ^ 1 is free: the products of the item before this one have completed
-          if (which == 1 && nv.n_tiles > 0 && nv.kind != kItemChain) { q_gather_start(nv, slot ^ 1); q_pending = true; }
+          const bool gather = which == 1 && nv.n_tiles > 0 && nv.kind != kItemChain;
+          if (gather) q_gather_start(nv, slot ^ 1);
           if (!stream_tiles(nv, 0, n_prefetched)) n_prefetched = 0;   // (aborting)
+          if (gather) {                        // published now: the Q K^T issuer starts on the next item before this one ends
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&C.q_full);
+          }
         }
       }
     } else if (warp == kSoftmaxWarps + 2) {
       // =================================================== S = Q K^T issuer ====================================
-      if (n_tiles > 0 && elect_one()) {                          // (elected, not `lane == 0`: see the producers)
+      // After the products of this item the warp goes straight on with the first kPreIssue products of the NEXT item
+      // (its Q rows and first K tiles were requested during this item): they run on the tensor pipe while the softmax
+      // warps finish this item and write its rows out, and the next item finds its first scores waiting.
+      int pre_next = 0;
+      if (elect_one()) {                                         // (elected, not `lane == 0`: see the producers)
         constexpr uint32_t idesc_qk = instr_desc_bf16(128, kTile, false);
-        const uint64_t q_desc0 = smem_desc_sw128(smem_u32(smem + kOffQ + slot * 32768), 0, 1024);
         const uint64_t k_desc0 = smem_desc_sw128(smem_u32(smem + kOffK), 0, 2048);   // 8-key groups 2048 B apart
-        bool ok = it.kind == kItemChain ? mbar_wait(&C.q_full_tma, q_uses_tma & 1, abort_flag)
-                                        : mbar_wait(&C.q_full, (q_uses - q_uses_tma) & 1, abort_flag);
-        for (int j = 0; j < n_tiles && ok; ++j) {
-          const uint32_t gj = g_tile + j;
+        // product of global tile gj with the Q rows in buffer `qbuf`; S buffer gj % kRing held S / P of tile
+        // gj - kRing and is free once the P V product that read it has completed
+        auto issue_qk = [&](uint32_t gj, int qbuf) -> bool {
           const int s = gj % kStagesK, b = gj % kRing;
-          // buffer b held S / P of tile j - kRing: free once the P V product that read it has completed
-          if (j >= kRing) ok = mbar_wait(&C.pv_done[b], ((gj - kRing) / kRing) & 1, abort_flag);
+          bool ok = gj < static_cast<uint32_t>(kRing) || mbar_wait(&C.pv_done[b], ((gj - kRing) / kRing) & 1, abort_flag);
           ok = ok && mbar_wait(&C.k_full[s], (gj / kStagesK) & 1, abort_flag);
-          if (!ok) break;
+          if (!ok) return false;
           tc_fence_after();
+          const uint64_t q_desc0 = smem_desc_sw128(smem_u32(smem + kOffQ + qbuf * 32768), 0, 1024);
           const uint64_t k_desc = smem_desc_advance(k_desc0, static_cast<uint32_t>(s) * kStageBytes);
           const uint32_t d_tmem = tmem + kColS + b * kTile;
 #pragma unroll
@@ -639,8 +687,32 @@ tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const _
                         kk > 0 ? 1u : 0u);
           mma_commit(&C.k_empty[s]);
           mma_commit(&C.s_full[b]);
+          return true;
+        };
+        bool ok = true;
+        if (n_tiles > qk_pre) {
+          ok = it.kind == kItemChain ? mbar_wait(&C.q_full_tma, q_uses_tma & 1, abort_flag)
+                                     : mbar_wait(&C.q_full, (q_uses - q_uses_tma) & 1, abort_flag);
+          for (int j = qk_pre; j < n_tiles && ok; ++j) ok = issue_qk(g_tile + j, slot);
+        }
+        if (ok && mbar_wait(&C.item_ready[slot ^ 1], ((item_seq + 1) >> 1) & 1, abort_flag)) {
+          const int e_next = C.item_e[slot ^ 1];
+          if (e_next >= 0 && e_next < n_items) {
+            const ItemView nv = view(C.item[slot ^ 1]);
+            if (nv.n_tiles > 0) {
+              const uint32_t used = n_tiles > 0 ? 1u : 0u;
+              const uint32_t qn = q_uses + used, qn_tma = q_uses_tma + ((used && it.kind == kItemChain) ? 1u : 0u);
+              ok = nv.kind == kItemChain ? mbar_wait(&C.q_full_tma, qn_tma & 1, abort_flag)
+                                         : mbar_wait(&C.q_full, (qn - qn_tma) & 1, abort_flag);
+              for (int j = 0; j < min(kPreIssue, nv.n_tiles) && ok; ++j) {
+                ok = issue_qk(g_tile + n_tiles + j, slot ^ 1);
+                if (ok) pre_next = j + 1;
+              }
+            }
+          }
         }
       }
+      qk_pre = __reduce_max_sync(0xffffffffu, pre_next);         // (the elected lane may differ from item to item)
     } else {
       // =================================================== O += P V issuer =====================================
       if (n_tiles > 0 && elect_one()) {
@@ -666,10 +738,16 @@ tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const _
         }
       }
     }
+#ifdef SS_STAMPS
+    if (tid == 0) { const long long t = clock64(); acc_epi += t - t_mark; t_mark = t; }
+#endif
     // ---- item end: every role meets here, so the next item starts from a drained pipeline --------------------
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+#ifdef SS_STAMPS
+    if (tid == 0) { const long long t = clock64(); acc_sync += t - t_mark; ++acc_items; }
+#endif
     // Exact second pass: the exponentials of some half-row overflowed the range of the lagged reference (scores that
     // rise by more than 2^40 from one tile to the next; the tensor-core pass has then written garbage for the
     // item).  All twelve warps recompute the item's rows on the CUDA cores, one row per warp and key by key.
@@ -696,6 +774,22 @@ tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const _
   }
   if (warp == kSoftmaxWarps) tmem_dealloc(tmem, kTmemCols);
   SS_STAMP_END(P.hdr, 3);
+#ifdef SS_STAMPS
+  if (tid == 0) {
+    atomicAdd(&P.hdr->stamp[8], static_cast<unsigned long long>(acc_first_s));
+    atomicAdd(&P.hdr->stamp[9], static_cast<unsigned long long>(acc_tiles));
+    atomicAdd(&P.hdr->stamp[10], static_cast<unsigned long long>(acc_o_wait));
+    atomicAdd(&P.hdr->stamp[11], static_cast<unsigned long long>(acc_epi));
+    atomicAdd(&P.hdr->stamp[12], static_cast<unsigned long long>(acc_sync));
+    atomicAdd(&P.hdr->stamp[13], static_cast<unsigned long long>(acc_items));
+    atomicAdd(&P.hdr->stamp[14], static_cast<unsigned long long>(tl_wait));
+    atomicAdd(&P.hdr->stamp[15], static_cast<unsigned long long>(tl_ld));
+    atomicAdd(&P.hdr->stamp[16], static_cast<unsigned long long>(tl_ref));
+    atomicAdd(&P.hdr->stamp[17], static_cast<unsigned long long>(tl_exp));
+    atomicAdd(&P.hdr->stamp[18], static_cast<unsigned long long>(tl_store));
+    atomicAdd(&P.hdr->stamp[19], static_cast<unsigned long long>(tl_tiles));
+  }
+#endif
 }
 
 }  // namespace split

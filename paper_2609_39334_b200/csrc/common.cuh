@@ -83,6 +83,18 @@ __device__ __forceinline__ void grid_dependency_enter() {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");
 }
+// Two variants for a pair of kernels that may overlap.  The EARLIER kernel of the pair enters with
+// grid_dependency_enter_then_release(): it waits for its own predecessor first and only then lets its successor be
+// scheduled, so the successor's blocks cannot start before that predecessor's results are complete.  The LATER kernel
+// enters with grid_dependency_release() alone, works on what does not depend on the earlier kernel, and calls
+// grid_dependency_wait() before it first touches the earlier kernel's results - and, in every thread, before it
+// exits, so that the kernel after it still sees plain stream order.
+__device__ __forceinline__ void grid_dependency_enter_then_release() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__device__ __forceinline__ void grid_dependency_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
