@@ -61,6 +61,63 @@ __device__ int block_excl_scan_chunks(int32_t* a, int n) {
   return total_s;
 }
 
+// Four independent scans of equal length in one pass (same scheme, one set of barriers): for the per-path arrays of
+// the one-block planner, where a scan is three barrier round trips and little else.
+__device__ void block_excl_scan4_chunks(int32_t* a0, int32_t* a1, int32_t* a2, int32_t* a3, int n, int (&total)[4]) {
+  __shared__ int warp_tot4[32][4];
+  __shared__ int total4_s[4];
+  int32_t* a[4] = {a0, a1, a2, a3};
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  const int chunk = (n + blockDim.x - 1) / blockDim.x;
+  const int lo = min(n, static_cast<int>(threadIdx.x) * chunk), hi = min(n, lo + chunk);
+  __syncthreads();
+  int sum[4], x[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    sum[k] = 0;
+    for (int i = lo; i < hi; ++i) sum[k] += a[k][i];
+    x[k] = sum[k];
+  }
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int y = __shfl_up_sync(0xffffffffu, x[k], o);
+      if (lane >= o) x[k] += y;
+    }
+  }
+  if (lane == 31) {
+#pragma unroll
+    for (int k = 0; k < 4; ++k) warp_tot4[warp][k] = x[k];
+  }
+  __syncthreads();
+  if (warp == 0) {
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      int t = lane < nw ? warp_tot4[lane][k] : 0;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int y = __shfl_up_sync(0xffffffffu, t, o);
+        if (lane >= o) t += y;
+      }
+      warp_tot4[lane][k] = t;
+      if (lane == 31) total4_s[k] = t;
+    }
+  }
+  __syncthreads();
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    int run = (warp ? warp_tot4[warp - 1][k] : 0) + x[k] - sum[k];
+    for (int i = lo; i < hi; ++i) {
+      const int v = a[k][i];
+      a[k][i] = run;
+      run += v;
+    }
+    total[k] = total4_s[k];
+  }
+  __syncthreads();
+}
+
 // The same scan for an array in GLOBAL memory: it goes through the block's staging buffer in shared memory when it
 // fits (coalesced in, scanned on chip, coalesced out) - every thread walking its own contiguous chunk of a global
 // array makes each load touch 32 different sectors, which cost the one-block scan kernel most of its time.
@@ -187,15 +244,26 @@ __device__ __forceinline__ void plan_scan_phase(const Params& P, int32_t* stage)
   const int tpt = P.tok_per_tile;
   if (tid == 0) s_total_tiles = 0;
 
-  // decode ranks
+#ifdef SS_STAMPS
+  long long pt = clock64();
+  int pi = 24;
+#define PLAN_MARK() do { __syncthreads(); if (tid == 0) { const long long t = clock64(); hdr->stamp[pi] = t - pt; pt = t; } ++pi; } while (0)
+#else
+#define PLAN_MARK() do { } while (0)
+#endif
+  // decode ranks (the one-block planner scans them together with the per-path counts below)
+  const bool fused = stage == nullptr;
   for (int p = tid; p < live; p += nt) P.path_dec_rank[p] = (P.path_class[p] == kClassDecode) ? 1 : 0;
-  const int n_dec = block_excl_scan(P.path_dec_rank, live, stage);
-  if (tid == 0) {
-    P.path_dec_rank[live] = n_dec;
-    hdr->n_dec = n_dec;
-    if (n_dec > P.caps.dec) set_status(&hdr->status, SS_ERR_WORKSPACE_TOO_SMALL);
+  if (!fused) {
+    const int n_dec = block_excl_scan(P.path_dec_rank, live, stage);
+    if (tid == 0) {
+      P.path_dec_rank[live] = n_dec;
+      hdr->n_dec = n_dec;
+      if (n_dec > P.caps.dec) set_status(&hdr->status, SS_ERR_WORKSPACE_TOO_SMALL);
+    }
   }
 
+  PLAN_MARK();   // 8: decode ranks
   // nodes: role, tiles
   for (int n = tid; n < N; n += nt) {
     const int np = P.node_npaths[n];
@@ -210,6 +278,7 @@ __device__ __forceinline__ void plan_scan_phase(const Params& P, int32_t* stage)
     if (tiles) atomicAdd(&s_total_tiles, tiles);
   }
   if (block_failed(hdr)) return;
+  PLAN_MARK();   // 9: node tiles
   const int total_tiles = s_total_tiles * P.Hkv;
   for (int n = tid; n < N; n += nt) {
     const int nd = P.node_ndec[n], len = P.node_kv_len[n];
@@ -238,12 +307,15 @@ __device__ __forceinline__ void plan_scan_phase(const Params& P, int32_t* stage)
     P.node_item_base[n] = tiles * splits * P.Hkv;
   }
   __syncthreads();
+  PLAN_MARK();   // 10: splits
   for (int n = tid; n < N; n += nt) {
     int off = 0;
     for (int a = P.node_parent[n]; a >= 0; a = P.node_parent[a]) off += P.node_own_slots[a];
     P.node_level_off[n] = off;
   }
+  PLAN_MARK();   // 11: level offsets
   const int n_stacked = block_excl_scan(P.node_item_base, N, stage);
+  PLAN_MARK();   // 12: item base scan
   if (tid == 0) P.node_item_base[N] = n_stacked;
 
   // decode paths: partial slots, leaf items; chain paths: tile items
@@ -262,9 +334,25 @@ __device__ __forceinline__ void plan_scan_phase(const Params& P, int32_t* stage)
     P.path_leaf_base[p] = leaf_items;
     P.path_chain_base[p] = chain_items;
   }
-  const int n_slots = block_excl_scan(P.path_slot_base, live, stage);
-  const int n_leaf_items = block_excl_scan(P.path_leaf_base, live, stage);
-  const int n_chain = block_excl_scan(P.path_chain_base, live, stage);
+  PLAN_MARK();   // 13: per-path counts
+  int n_slots, n_leaf_items, n_chain;
+  if (fused) {
+    int tot[4];
+    block_excl_scan4_chunks(P.path_slot_base, P.path_leaf_base, P.path_chain_base, P.path_dec_rank, live, tot);
+    n_slots = tot[0];
+    n_leaf_items = tot[1];
+    n_chain = tot[2];
+    if (tid == 0) {
+      P.path_dec_rank[live] = tot[3];
+      hdr->n_dec = tot[3];
+      if (tot[3] > P.caps.dec) set_status(&hdr->status, SS_ERR_WORKSPACE_TOO_SMALL);
+    }
+  } else {
+    n_slots = block_excl_scan(P.path_slot_base, live, stage);
+    n_leaf_items = block_excl_scan(P.path_leaf_base, live, stage);
+    n_chain = block_excl_scan(P.path_chain_base, live, stage);
+  }
+  PLAN_MARK();   // 14: three scans
   if (tid == 0) {
     hdr->n_slots = n_slots;
     hdr->n_stacked_items = n_stacked;
@@ -415,7 +503,7 @@ constexpr int kSmallPlan = 2048;               // nodes and paths
 constexpr int kSmallNodeArrays = 11, kSmallPathArrays = 6;
 // bytes of shared memory for N nodes and NP paths: staged inputs + redirected plan arrays
 inline size_t small_plan_smem(int N, int NP) {
-  return static_cast<size_t>(N + 1) * (8 + 4 + 4 + 4 * kSmallNodeArrays) + static_cast<size_t>(NP + 1) * (4 + 4 + 4 * kSmallPathArrays) + 64;
+  return static_cast<size_t>(N + 1) * (8 + 4 + 4 + 4 * kSmallNodeArrays) + static_cast<size_t>(NP + 1) * (8 + 8 + 4 + 4 + 4 * kSmallPathArrays) + 64;
 }
 
 __global__ void __launch_bounds__(kScanThreads) plan_small_kernel(const Params P0) {
@@ -432,9 +520,11 @@ __global__ void __launch_bounds__(kScanThreads) plan_small_kernel(const Params P
   P.num_paths_dev = &s_live;
   __syncthreads();
   SS_STAMP_BEGIN(P.hdr, 0);
-  // carve: 8-byte array first, then 4-byte arrays of N + 1 and of NP + 1 entries
+  // carve: the 8-byte arrays first, then 4-byte arrays of N + 1 and of NP + 1 entries
   int64_t* s_page_off = reinterpret_cast<int64_t*>(plan_smem);
-  int32_t* w = reinterpret_cast<int32_t*>(s_page_off + (N + 1));
+  int64_t* s_q_off = s_page_off + (N + 1);
+  int64_t* s_q_src = s_q_off + (NP + 1);
+  int32_t* w = reinterpret_cast<int32_t*>(s_q_src + (NP + 1));
   auto take = [&](int n) { int32_t* p = w; w += n; return p; };
   int32_t* s_parent = take(N + 1);
   int32_t* s_len = take(N + 1);
@@ -452,6 +542,14 @@ __global__ void __launch_bounds__(kScanThreads) plan_small_kernel(const Params P
   for (int n = tid; n <= N; n += nt) s_page_off[n] = P0.node_page_offsets[n];
   const int live = s_live;
   for (int p = tid; p < live; p += nt) { s_leaf[p] = P0.path_leaf_node[p]; s_qlen[p] = P0.path_q_len[p]; }
+  // (the row offsets too: the emission reads them per ITEM, and a global load behind each binary search was half of
+  //  its time)
+  for (int p = tid; p <= live; p += nt) s_q_off[p] = P0.q_offsets[p];
+  if (P0.q_src_offsets) {
+    for (int p = tid; p < live; p += nt) s_q_src[p] = P0.q_src_offsets[p];
+    P.q_src_offsets = s_q_src;
+  }
+  P.q_offsets = s_q_off;
   P.node_parent = s_parent;
   P.node_kv_len = s_len;
   P.node_page_offsets = s_page_off;
@@ -459,16 +557,27 @@ __global__ void __launch_bounds__(kScanThreads) plan_small_kernel(const Params P
   P.path_q_len = s_qlen;
   __syncthreads();
 
+#ifdef SS_STAMPS
+  long long small_t = clock64();
+#define SMALL_MARK(i) do { __syncthreads(); if (tid == 0) { const long long t = clock64(); s_hdr.stamp[i] = t - small_t; small_t = t; } } while (0)
+#else
+#define SMALL_MARK(i) do { } while (0)
+#endif
+  SMALL_MARK(32);                                    // staging of the inputs
   plan_nodes_phase(P);
   bool failed = block_failed(P.hdr);
+  SMALL_MARK(33);
   if (!failed) {
     plan_paths_phase(P);
     __syncthreads();
+    SMALL_MARK(34);
     plan_scan_phase(P, nullptr);                     // (the arrays are in shared memory already)
     failed = block_failed(P.hdr);
+    SMALL_MARK(35);
   }
   if (!failed) {
     plan_emit_phase(P);
+    SMALL_MARK(36);
     // the executors read these three from the workspace (exact second pass, generic rows)
     for (int n = tid; n < N; n += nt) P0.node_start[n] = P.node_start[n];
     for (int p = tid; p < live; p += nt) { P0.path_class[p] = P.path_class[p]; P0.path_kv_len[p] = P.path_kv_len[p]; }
@@ -516,7 +625,9 @@ int32_t launch_plan(const Params& P, cudaStream_t st) {
     }
   }
   SS_LAUNCH(plan_scan_kernel, 1, kScanThreads, kScanStage * 4, st, P);
-  SS_LAUNCH(plan_emit_kernel, blocks, kGridThreads, 0, st, P);
+  // one thread per ITEM (there are an order of magnitude more items than paths; their number is known on the device
+  // only): a grid that covers the typical item count in one or two strides
+  SS_LAUNCH(plan_emit_kernel, blocks < 64 ? 8 * blocks : 1184, kGridThreads, 0, st, P);
   return SS_OK;
 }
 

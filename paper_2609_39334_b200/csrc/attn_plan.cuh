@@ -66,7 +66,7 @@ struct PlanHeader {       // first bytes of the workspace; status MUST be the fi
   int32_t n_stacked_items; // tile items [0, n_stacked_items) are stacked items, the rest chain items
   int32_t pad[6];
 #ifdef SS_STAMPS
-  unsigned long long stamp[24];  // instrumented build: %globaltimer at kernel starts / ends (see SS_STAMP); 8..23:
+  unsigned long long stamp[40];  // instrumented build: %globaltimer at kernel starts / ends (see SS_STAMP); 8..23 (24..31: phases of the planner's scan; 32..36: of the one-block planner):
                                  // clock sums of one softmax thread per tile-kernel block (where an item's time goes)
 #endif
 };
