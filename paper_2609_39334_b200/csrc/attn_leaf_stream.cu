@@ -1,8 +1,9 @@
 // Decode-leaf attention, streaming version (the default): bandwidth-bound, so what counts is bytes in flight.
 // Every warp is a pipeline of its own: an elected lane streams the (page, kv head) blocks of K and V of the warp's
-// leaf items through a private ring of shared memory with bulk-tensor copies (4 pages = 32 KB in flight per warp,
-// ~190 KB per SM, three times what a register-staged loop can hold), and the warp consumes them with ldmatrix +
-// mma.sync.m16n8k16 (the G query rows of the GQA group padded to 16; fp32 online softmax in the exp2 domain with quad
+// leaf items through a private ring of shared memory with bulk-tensor copies (2 pages = 16 KB in flight per warp,
+// 12 warps: ~190 KB per SM, three times what a register-staged loop can hold; groups of 9-16 query heads: 8 warps x
+// 3 pages), and the warp consumes them with ldmatrix + mma.sync.m16n8k16 in transposed form (the 16 keys of a page
+// are the M dimension, the query rows of the GQA group the N dimension; fp32 online softmax in the exp2 domain with
 // shuffles).  The copies use the same tensor map as the tile kernel (each block lands as 128-byte-swizzled 8-row
 // atoms), so the ldmatrix reads are free of bank conflicts.  Items are taken from a global counter; the NEXT item's
 // descriptor, page ids and query rows are fetched while the current item is computed and its pages are requested as
@@ -10,8 +11,8 @@
 //
 // The kernel also finishes the decode tokens: an item writes its normalised fp32 partial (o, lse), counts itself in
 // leaf_arrive[token][kv head], and the warp that brings the count to the token's number of leaf chunks merges ALL
-// partials of that (token, kv head) - the shared-node partials were written by the tile kernel, which is complete
-// before this kernel starts - and writes the final bf16 rows.  Tokens without a private leaf, and rows of GENERIC
+// partials of that (token, kv head) - the shared-node partials come from the tile kernel, for whose completion a
+// warp waits before its first read of them - and writes the final bf16 rows.  Tokens without a private leaf, and rows of GENERIC
 // paths, are swept after the items.  No separate merge launch.
 #include "attn_plan.cuh"
 #include "attn_rows.cuh"

@@ -3,9 +3,10 @@
 // attn_umma.cu (a 64-key tile there); what differs follows from measurements on this part:
 //   * an SM retires one tcgen05 instruction (MMA or commit) per ~50 clocks whatever its shape, and a 64-key tile costs
 //     17 of them: with 128-key tiles every MMA is M128 x N128 x K16 (64 clocks of math) and the count per key halves;
-//   * an ex2 holds an SM sub-partition for 8 clocks and every other instruction issued there ADDS to that (the pipes
-//     do not overlap in issue), so the loop works on packed fp32 pairs, takes the row maximum from a sample of the
-//     columns inside the exponential loop, and uses a reference maximum that lags one tile behind;
+//   * an ex2 occupies the special-function unit of an SM sub-partition for 8 clocks, and in the dependent chain of the
+//     softmax loop (scale, exponential, sum, convert; 168 registers leave little room to interleave pairs) nearly
+//     every other instruction adds to that, so the loop works on packed fp32 pairs, takes the row maximum from a
+//     sample of the columns inside the exponential loop, and uses a reference maximum that lags one tile behind;
 //   * a score buffer is recycled only when the P V product that read it has completed, so with two buffers the chain
 //     Q K^T -> softmax -> P V of one tile bounds the next but one: three S/P buffers (128 columns each) + O (128
 //     columns) fill the TMEM exactly, Q stays in shared memory;
@@ -27,7 +28,8 @@
 // from TMEM, V MN-major); lane 1 of warp 11 fetches the NEXT item while this one runs: the producers then load its
 // first K / V tiles and its Q rows (a 3-D TMA box for a chain item, issued by the K producer; cp.async of the
 // gathered rows of a stacked item by the V producer warp) into the second Q buffer before the current item has
-// drained.  The softmax warps do nothing but the softmax and the epilogue.
+// drained, and the Q K^T issuer goes on with the next item's first two products as soon as it has issued the current
+// item's last.  The softmax warps do nothing but the softmax and the epilogue.
 // Every wait is bounded; on expiry the CTA raises its abort flag, the later waits fail fast, the roles run through
 // the item's remaining tiles without writing results, the CTA frees its TMEM and the kernel records SS_ERR_TIMEOUT.
 #include "attn_plan.cuh"
