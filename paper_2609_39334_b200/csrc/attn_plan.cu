@@ -118,6 +118,89 @@ __device__ void block_excl_scan4_chunks(int32_t* a0, int32_t* a1, int32_t* a2, i
   __syncthreads();
 }
 
+// The same for arrays in GLOBAL memory of up to 16 entries per thread: a thread keeps its 16 consecutive entries of
+// each array in registers (128-bit loads, all issued before the first is used; 128-bit stores), so a pair of scans
+// costs two trips to memory instead of the six of two staged scans.  The arrays must be 16-byte aligned.
+constexpr int kScanRegs = 16;
+__device__ void block_excl_scan2_regs(int32_t* a0, int32_t* a1, int n, int (&total)[2]) {   // (two arrays per call: 32 of a thread's 64 registers)
+  __shared__ int warp_tot4[32][2];
+  __shared__ int total4_s[2];
+  int32_t* a[2] = {a0, a1};
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  const int lo = static_cast<int>(threadIdx.x) * kScanRegs;
+  int v[2][kScanRegs];
+  __syncthreads();
+#pragma unroll
+  for (int k = 0; k < 2; ++k) {
+#pragma unroll
+    for (int i = 0; i < kScanRegs; i += 4) {
+      if (lo + i + 4 <= n) {
+        const int4 q = *reinterpret_cast<const int4*>(a[k] + lo + i);
+        v[k][i] = q.x; v[k][i + 1] = q.y; v[k][i + 2] = q.z; v[k][i + 3] = q.w;
+      } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) v[k][i + j] = (lo + i + j < n) ? a[k][lo + i + j] : 0;
+      }
+    }
+  }
+  int sum[2], x[2];
+#pragma unroll
+  for (int k = 0; k < 2; ++k) {
+    sum[k] = 0;
+#pragma unroll
+    for (int i = 0; i < kScanRegs; ++i) sum[k] += v[k][i];
+    x[k] = sum[k];
+  }
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      const int y = __shfl_up_sync(0xffffffffu, x[k], o);
+      if (lane >= o) x[k] += y;
+    }
+  }
+  if (lane == 31) {
+#pragma unroll
+    for (int k = 0; k < 2; ++k) warp_tot4[warp][k] = x[k];
+  }
+  __syncthreads();
+  if (warp == 0) {
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      int t = lane < nw ? warp_tot4[lane][k] : 0;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int y = __shfl_up_sync(0xffffffffu, t, o);
+        if (lane >= o) t += y;
+      }
+      warp_tot4[lane][k] = t;
+      if (lane == 31) total4_s[k] = t;
+    }
+  }
+  __syncthreads();
+#pragma unroll
+  for (int k = 0; k < 2; ++k) {
+    int run = (warp ? warp_tot4[warp - 1][k] : 0) + x[k] - sum[k];
+#pragma unroll
+    for (int i = 0; i < kScanRegs; i += 4) {
+      int4 q;
+      q.x = run; run += v[k][i];
+      q.y = run; run += v[k][i + 1];
+      q.z = run; run += v[k][i + 2];
+      q.w = run; run += v[k][i + 3];
+      if (lo + i + 4 <= n) {
+        *reinterpret_cast<int4*>(a[k] + lo + i) = q;
+      } else {
+        if (lo + i < n) a[k][lo + i] = q.x;
+        if (lo + i + 1 < n) a[k][lo + i + 1] = q.y;
+        if (lo + i + 2 < n) a[k][lo + i + 2] = q.z;
+      }
+    }
+    total[k] = total4_s[k];
+  }
+  __syncthreads();
+}
+
 // The same scan for an array in GLOBAL memory: it goes through the block's staging buffer in shared memory when it
 // fits (coalesced in, scanned on chip, coalesced out) - every thread walking its own contiguous chunk of a global
 // array makes each load touch 32 different sectors, which cost the one-block scan kernel most of its time.
@@ -251,8 +334,11 @@ __device__ __forceinline__ void plan_scan_phase(const Params& P, int32_t* stage)
 #else
 #define PLAN_MARK() do { } while (0)
 #endif
-  // decode ranks (the one-block planner scans them together with the per-path counts below)
-  const bool fused = stage == nullptr;
+  // decode ranks (scanned together with the per-path counts below where one pass can take all four arrays)
+  const bool fused_regs = stage != nullptr && live <= nt * kScanRegs &&
+                          ((reinterpret_cast<uintptr_t>(P.path_slot_base) | reinterpret_cast<uintptr_t>(P.path_leaf_base) |
+                            reinterpret_cast<uintptr_t>(P.path_chain_base) | reinterpret_cast<uintptr_t>(P.path_dec_rank)) & 15) == 0;
+  const bool fused = stage == nullptr || fused_regs;
   for (int p = tid; p < live; p += nt) P.path_dec_rank[p] = (P.path_class[p] == kClassDecode) ? 1 : 0;
   if (!fused) {
     const int n_dec = block_excl_scan(P.path_dec_rank, live, stage);
@@ -338,7 +424,15 @@ __device__ __forceinline__ void plan_scan_phase(const Params& P, int32_t* stage)
   int n_slots, n_leaf_items, n_chain;
   if (fused) {
     int tot[4];
-    block_excl_scan4_chunks(P.path_slot_base, P.path_leaf_base, P.path_chain_base, P.path_dec_rank, live, tot);
+    if (fused_regs) {
+      int t2[2];
+      block_excl_scan2_regs(P.path_slot_base, P.path_leaf_base, live, t2);
+      tot[0] = t2[0];
+      tot[1] = t2[1];
+      block_excl_scan2_regs(P.path_chain_base, P.path_dec_rank, live, t2);
+      tot[2] = t2[0];
+      tot[3] = t2[1];
+    } else block_excl_scan4_chunks(P.path_slot_base, P.path_leaf_base, P.path_chain_base, P.path_dec_rank, live, tot);
     n_slots = tot[0];
     n_leaf_items = tot[1];
     n_chain = tot[2];

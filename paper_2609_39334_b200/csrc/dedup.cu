@@ -412,7 +412,7 @@ small_match_finalize_kernel(const uint32_t* __restrict__ keys, const uint32_t* _
 // One block.  Thread t owns kGatherItems consecutive unique paths per round: it gathers their descriptor rows and the
 // block scans the query lengths (thread sums -> warp shuffles -> warp totals -> running carry).
 constexpr int kGatherThreads = 1024;
-constexpr int kGatherItems = 4;
+constexpr int kGatherItems = 4;       // (16 per thread - one round for 16384 paths - was measured: 33 -> 60 us, every access 32 sectors wide)
 
 __global__ void __launch_bounds__(kGatherThreads)
 gather_unique_kernel(const int32_t* __restrict__ unique_paths, const int32_t* __restrict__ num_unique, int n,
