@@ -136,9 +136,12 @@ class ClockSampler:
 # ------------------------------------------------------------------------------------------------------------
 # CPU oracle arm (cpu_baseline leg and --impl reference)
 # ------------------------------------------------------------------------------------------------------------
-def oracle_sample(w, seed=0):
+def oracle_sample(w, seed=0, budget_scale=1.0, min_paths=None):
     """A bounded sample of the workload for the CPU oracle: a few verification paths and more decode paths,
-    sized by the host core count for roughly 10-30 s of CPU work per pass."""
+    sized by the host core count for roughly 10-30 s of CPU work per pass (`budget_scale` shrinks that for a run of
+    many passes; `min_paths`: the least number of unique paths, MIN_ORACLE_SAMPLE unless given)."""
+    if min_paths is None:
+        min_paths = MIN_ORACLE_SAMPLE
     import oracle
     cores = oracle.host_cores()
     rng = np.random.default_rng(seed)
@@ -147,13 +150,13 @@ def oracle_sample(w, seed=0):
     T = w.path_q_len[uniq]
     ver, dec = uniq[T > 1], uniq[T == 1]
     # fp64 cost model: pairs * Hq * 2 * D multiply-adds; ~0.7 G mul-add/s per core for this plain loop
-    budget_pairs = 12.0 * cores * 0.7e9 / (2.0 * w.head_dim * w.num_q_heads)
+    budget_pairs = budget_scale * 12.0 * cores * 0.7e9 / (2.0 * w.head_dim * w.num_q_heads)
     chosen, pairs = [], 0.0
     pools = [list(rng.permutation(ver)), list(rng.permutation(dec))]
     turn = 0
     # one verification path, then three decode paths (a decode path costs 1/T of a verification path), until the
     # budget is spent AND at least MIN_ORACLE_SAMPLE unique paths are in
-    while (pools[0] or pools[1]) and (pairs < budget_pairs or len(chosen) < MIN_ORACLE_SAMPLE):
+    while (pools[0] or pools[1]) and (pairs < budget_pairs or len(chosen) < min_paths):
         pool = pools[0] if (turn % 4 == 0 and pools[0]) or not pools[1] else pools[1]
         turn += 1
         p = int(pool.pop())
@@ -444,7 +447,11 @@ def main():
         oracle.build()
         dev = "cuda:0" if torch.cuda.is_available() else "cpu"
         w = synth.make_config(cfg_idx, device=dev, scale=args.scale)
-        sample = oracle_sample(w)
+        # every step is one pass over a bounded sample; the sample shrinks with the number of passes so that the whole
+        # run stays within a few minutes (the default 10 + 1 passes: about a quarter of the single-pass sample each)
+        passes = max(args.steps, 1) + min(args.warmup, 1)
+        scale = min(1.0, 4.0 / passes)
+        sample = oracle_sample(w, budget_scale=scale, min_paths=MIN_ORACLE_SAMPLE if scale >= 1.0 else 32)
         sub = synth.extract_subworkload(w, sample)
         del w
         if dev != "cpu":
