@@ -406,6 +406,25 @@ def test_attention_page_permutation_and_explicit_scale():
     assert np.array_equal(r2["out"], r1["out"]) and np.array_equal(r2["lse"], r1["lse"])
 
 
+def test_attention_on_a_limited_number_of_sms_gives_the_same_result():
+    """`max_sms` only changes how many blocks the tile and leaf kernels launch (the host-buffer step keeps a few SMs for
+    its copy kernel): every item is computed by one block in the same order of operations, so the result is the same
+    to the bit, and a value above the device's SM count means all of them."""
+    w = synth.build_tree_workload("sms", 31, 12, 2, [256], [9], 3, (1, 600), lambda i, n, rng: 1 + (i % 3 == 0) * 40)
+    outs = []
+    for sms in (0, 3, 1, 100000):
+        pipe = DevicePipeline(w, DEV, attn_flags=B.SS_FLAG_VALIDATE)
+        pipe.desc.max_sms = sms
+        pipe.dedup()
+        pipe.compact_unique()
+        pipe.attention()
+        outs.append(pipe.results())
+    ref = oracle.dedup(w.tok_ids, w.tok_offsets, w.ctx_key, w.slot_in)
+    check_attention(outs[0], w, ref, max_paths=16)
+    for r in outs[1:]:
+        assert np.array_equal(r["out"], outs[0]["out"]) and np.array_equal(r["lse"], outs[0]["lse"])
+
+
 def test_attention_flat_per_path_page_tables():
     """A cache that keeps one flat page list per sequence is the tree form with one node per path: a root that is its
     own leaf, whose page list is the whole sequence.  Same pool, same queries: the results must agree with the oracle
