@@ -127,9 +127,18 @@ leaf_stream_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
   int f_e = 0;
   LeafItem f_it;
   uint32_t nq[NT][8][2];                                         // query fragments of the item being fetched
+  bool first_claim = true;
   auto fetch_claim = [&]() {                                     // step 1: claim an item index
+    // (a warp's first item is its own index in the grid - one trip to memory less before its first page - and the
+    //  counter hands out the items after those)
+    const int n_warps_grid = static_cast<int>(gridDim.x) * WARPS;
+    if (first_claim) {
+      f_e = static_cast<int>(blockIdx.x) * WARPS + warp;
+      first_claim = false;
+      return;
+    }
     int e = 0;
-    if (lane == 0) e = atomicAdd(&P.hdr->leaf_counter, 1);
+    if (lane == 0) e = atomicAdd(&P.hdr->leaf_counter, 1) + n_warps_grid;
     f_e = __shfl_sync(0xffffffffu, e, 0);
   };
   auto fetch_desc = [&]() {                                      // step 2: its descriptor

@@ -148,10 +148,11 @@ __device__ __noinline__ void exact_second_pass(const Params& P, const TileItem* 
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
                             const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ Params P) {
-  ss::grid_dependency_enter_then_release();   // (the leaf kernel behind this one starts without waiting for it)
+  // The block first sets up what needs nothing from the kernels before it (barriers, the zeroed Q buffers, tensor
+  // memory): launched with programmatic serialization it may be resident while the planner is still running, and
+  // this part then overlaps the planner's tail.  It waits for the planner right after (see below).
   extern __shared__ __align__(1024) uint8_t smem[];
   __shared__ Ctrl C;
-  SS_STAMP_BEGIN(P.hdr, 2);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   volatile int* abort_flag = &C.abort_flag;
 
@@ -180,6 +181,10 @@ tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const _
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  // ---- from here on the planner's results are read: wait for it, then let the leaf kernel behind this one start
+  //      (it needs the plan too, and nothing from this kernel until it merges)
+  ss::grid_dependency_enter_then_release();
+  SS_STAMP_BEGIN(P.hdr, 2);
   const uint32_t tmem = C.tmem_slot;
   const int n_items = P.hdr->n_tile_items;
   const int G = P.G;
@@ -196,9 +201,12 @@ tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const _
   uint32_t prod_wraps = 0;  //   (kept as counters: a modulo by a stage count that differs per warp is a division per tile)
 
   // Takes the next item from the global counter into slot `dst` (one thread).
-  auto fetch_item = [&](int dst) {
+  auto fetch_item = [&](int dst, bool first_fetch) {
+    // (a block's first item is its own index: no trip to the counter before the first tile; the counter hands out
+    //  the items after the first gridDim.x)
     int e = -1;
-    if (P.hdr->status == SS_OK && !C.abort_flag) e = atomicAdd(&P.hdr->tile_counter, 1);
+    if (P.hdr->status == SS_OK && !C.abort_flag)
+      e = first_fetch ? static_cast<int>(blockIdx.x) : atomicAdd(&P.hdr->tile_counter, 1) + static_cast<int>(gridDim.x);
     if (e >= 0 && e < n_items) C.item[dst] = P.tile_items[e];
     C.item_e[dst] = e;
     __threadfence_block();
@@ -237,7 +245,7 @@ tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const _
     tma_load_3d(dst + 16384, &tmap_q, 64, v.g * G, v.src0, &C.q_full_tma);
   };
 
-  if (tid == 0) fetch_item(0);
+  if (tid == 0) fetch_item(0, true);
   __syncthreads();
   bool q_pending = false;   // V producer warp: the gather of the first item's Q rows is under way
   int qk_pre = 0;           // Q K^T issuer warp: products of the coming item that were issued during the one before
@@ -274,7 +282,7 @@ tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const _
     if (e < 0 || e >= n_items) break;
     const ItemView it = view(C.item[slot]);
     const int n_tiles = it.n_tiles;
-    if (tid == (kSoftmaxWarps + 3) * 32 + 1) fetch_item(slot ^ 1);   // a lane that has nothing else to do
+    if (tid == (kSoftmaxWarps + 3) * 32 + 1) fetch_item(slot ^ 1, false);   // a lane that has nothing else to do
 
     if (warp < kSoftmaxWarps) {
       // =================================================== softmax + epilogue ==================================

@@ -134,6 +134,13 @@ def test_every_kernel_waits_for_its_predecessor_first():
             if not ok and "leaf_stream_kernel" in m.group(0):
                 body = rest[:rest.index("\n}\n")] if "\n}\n" in rest else rest
                 ok = "ss::grid_dependency_release();" in rest[:600] and rest.count("ss::grid_dependency_wait();") >= 3
+            if not ok and "tile_items_umma_split_kernel" in m.group(0):
+                # block-local setup first (barriers, zeroed buffers, tensor memory), then the wait - before anything of
+                # the plan is read
+                body = rest[:rest.index("\n}\n")] if "\n}\n" in rest else rest
+                at = body.find("ss::grid_dependency_enter_then_release();")
+                first_plan_read = min(x for x in (body.find("P.hdr"), body.find("P.tile_items"), len(body)) if x >= 0)
+                ok = 0 <= at < first_plan_read
             assert ok, (os.path.basename(path), m.group(0)[:80])
         assert "<<<" not in src, path            # every launch goes through the counting macro
     assert n >= 20
