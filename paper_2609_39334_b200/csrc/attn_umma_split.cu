@@ -295,12 +295,11 @@ tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const _
       const int i = row / G, hl = row - i * G;
       const bool row_valid = i < it.n_tok;
       const int h = it.g * G + hl;
-      int64_t q_row = 0;                                          // output row
-      int dec = 0;
-      if (row_valid) {
-        if (it.kind == kItemChain) q_row = it.tok0 + i;
-        else { dec = it.tok0 + i; q_row = P.dec_tok[dec]; }
-      }
+      // where the row goes: the output row of a chain item's token, the partial slot of a stacked item's token (read
+      // now, so that the load is long done when the epilogue needs it)
+      int64_t out_row = 0;
+      if (row_valid) out_row = it.kind == kItemChain ? static_cast<int64_t>(it.tok0 + i)
+                                                     : static_cast<int64_t>(P.dec_slot_base[it.tok0 + i]) + it.slot_off;
       const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
       auto pair_barrier = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(2 + (warp & 3)) : "memory"); };
       float m = 0.f, l = 0.f;                                     // reference maximum (0 while the row has no visible key)
@@ -489,8 +488,7 @@ tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const _
       C.xmax[0][hf][row] = 0u;
 #ifdef SS_CHECKED
       {                                                           // (warp-uniform outcome: the loads below are collective)
-        const bool in_range = !row_valid || (it.slot_off < 0 ? (q_row >= 0 && q_row < P.total_q)
-                                                             : (static_cast<int64_t>(P.dec_slot_base[dec]) + it.slot_off < P.caps.slots));
+        const bool in_range = !row_valid || (out_row >= 0 && out_row < (it.slot_off < 0 ? P.total_q : static_cast<int64_t>(P.caps.slots)));
         if (!in_range) set_status(&P.hdr->status, SS_ERR_BAD_INPUT);
         if (!__all_sync(0xffffffffu, in_range)) ok = false;
       }
@@ -499,7 +497,6 @@ tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const _
         const float inv = l_all > 0.f ? 1.f / l_all : 0.f;
         const float lse = l_all > 0.f ? m * P.scale + __logf(l_all) : -INFINITY;
         const bool final_out = it.slot_off < 0;
-        const int64_t slot_row = final_out ? 0 : static_cast<int64_t>(row_valid ? P.dec_slot_base[dec] : 0) + it.slot_off;
 #pragma unroll
         for (int c0 = hf * 64; c0 < hf * 64 + 64; c0 += 32) {
           uint32_t orow[32];
@@ -513,7 +510,7 @@ tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const _
           }
           if (!row_valid) continue;
           if (final_out) {
-            __nv_bfloat16* dst = P.out + (q_row * P.Hq + h) * kHeadDim + c0;
+            __nv_bfloat16* dst = P.out + (out_row * P.Hq + h) * kHeadDim + c0;
 #pragma unroll
             for (int x = 0; x < 2; ++x) {
               uint32_t w[8];
@@ -523,7 +520,7 @@ tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const _
               st_global_32B(dst + 16 * x, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]);
             }
           } else {
-            float* dst = P.part_o + (slot_row * P.Hq + h) * kHeadDim + c0;
+            float* dst = P.part_o + (out_row * P.Hq + h) * kHeadDim + c0;
 #pragma unroll
             for (int x = 0; x < 4; ++x) {
               uint32_t w[8];
@@ -534,8 +531,8 @@ tile_items_umma_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const _
           }
         }
         if (row_valid && hf == 0) {
-          if (final_out) { if (P.lse) P.lse[q_row * P.Hq + h] = lse; }
-          else P.part_lse[slot_row * P.Hq + h] = lse;
+          if (final_out) { if (P.lse) P.lse[out_row * P.Hq + h] = lse; }
+          else P.part_lse[out_row * P.Hq + h] = lse;
         }
       }
     } else if (warp < kSoftmaxWarps + 2) {
